@@ -1,0 +1,201 @@
+/*
+ * CPU fp64 oracle for the draft-tree verification step.  TEST INFRASTRUCTURE ONLY:
+ * it is called by the tests, by the smoke check and by the benchmark's CPU-baseline
+ * leg, never by the product path, and it shares no source with the CUDA library.
+ *
+ * Everything here is the plain definition written out, with no blocking, fusion or
+ * reordering, so that it can be checked against the paper by eye:
+ *
+ *   oracle_tree_mask    ancestor sets of a draft tree (the tree of Sec. 3.1, "context-aware
+ *                       dynamic draft tree"; the mask itself is standard tree decoding
+ *                       mechanics the paper inherits by citation)
+ *   oracle_tree_attn    softmax attention of Eq. 1 (with the 1/sqrt(d) scale Eq. 1 drops
+ *                       "for simplicity" restored as an explicit argument), restricted per
+ *                       tree node to the committed prefix plus the node's ancestors
+ *   oracle_accept       the acceptance rule of Sec. 3.1 at temperature 0 (Table 1, upper
+ *                       half): a drafted token survives iff it equals the target's greedy
+ *                       token at its parent; the result is the longest surviving root path
+ *   oracle_kv_compact   commit of the accepted rows into the pre-allocated cache (App. A)
+ *
+ * Layouts (row-major, C order):
+ *   q, out            [B, N, Hq, D]
+ *   k_cache, v_cache  [B, Hkv, S_max, D]   bf16 carried as uint16 bit patterns
+ *   tree_mask         [B, N, W] uint64, W = ceil(N/64); bit t of row i <=> node t visible to node i
+ *   parents, ids      [B, N] int32; parents[b][0] = -1
+ *   path              [B, N] int32 padded with -1
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_f64(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Ancestor mask: bit t of mask[b][i] is set iff t is i itself or is reached from i by following
+ * parent links up to the root.  depth[b][i] = number of links from i to the root.
+ * Returns 0, or -1 if some parent is not an earlier node (the row is still written: self bit only). */
+int oracle_tree_mask(const int32_t* parents, int B, int N, uint64_t* mask, int32_t* depth) {
+    int W = (N + 63) / 64, bad = 0;
+    for (int b = 0; b < B; ++b) {
+        const int32_t* par = parents + (size_t)b * N;
+        for (int i = 0; i < N; ++i) {
+            uint64_t* row = mask + ((size_t)b * N + i) * W;
+            for (int w = 0; w < W; ++w) row[w] = 0;
+            int ok = (par[0] == -1);
+            for (int a = i; ok && a != 0; a = par[a])      /* every link must point to an earlier node */
+                if (par[a] < 0 || par[a] >= a) ok = 0;
+            int d = 0;
+            if (!ok) {
+                bad = 1;
+                row[i / 64] |= (uint64_t)1 << (i % 64);
+            } else {
+                for (int a = i; a != -1; a = par[a]) {
+                    row[a / 64] |= (uint64_t)1 << (a % 64);
+                    if (par[a] != -1) ++d;
+                }
+            }
+            if (depth) depth[(size_t)b * N + i] = d;
+        }
+    }
+    return bad ? -1 : 0;
+}
+
+/* Tree-masked attention, Eq. 1 with scale.  For sequence b, query head h (kv head h / G) and tree
+ * node i the allowed key set is A = { j : j < S } U { S + t : bit t of tree_mask[b][i] }, S = kv_len[b]:
+ *     s_j = scale * <q, k_j>,  alpha_j = exp(s_j) / sum_{A} exp(s_k),  out = sum_{A} alpha_j v_j.
+ * The maximum is subtracted before exponentiation (it cancels in alpha).  out is fp64;
+ * lse[b][h][i] = log sum_A exp(s_j) (may be NULL).  An empty A gives out = 0, lse = -inf. */
+int oracle_tree_attn(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache,
+                     const int32_t* kv_len, const uint64_t* tree_mask,
+                     int B, int N, int Hq, int Hkv, int D, int S_max, double scale,
+                     double* out, double* lse) {
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    int G = Hq / Hkv, W = (N + 63) / 64;
+    for (int b = 0; b < B; ++b)
+        if (kv_len[b] < 0 || kv_len[b] + N > S_max) return -2;
+    int status = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < Hq; ++h) {
+            int S = kv_len[b], kvh = h / G;
+            const uint16_t* Kh = k_cache + ((size_t)b * Hkv + kvh) * (size_t)S_max * D;
+            const uint16_t* Vh = v_cache + ((size_t)b * Hkv + kvh) * (size_t)S_max * D;
+            double* s = (double*)malloc(sizeof(double) * (size_t)(S + N));
+            unsigned char* allowed = (unsigned char*)malloc((size_t)(S + N));
+            double* qd = (double*)malloc(sizeof(double) * (size_t)D);
+            if (!s || !allowed || !qd) { status = -3; free(s); free(allowed); free(qd); continue; }
+            for (int i = 0; i < N; ++i) {
+                const uint16_t* qi = q + (((size_t)b * N + i) * Hq + h) * D;
+                const uint64_t* mrow = tree_mask + ((size_t)b * N + i) * W;
+                double* o = out + (((size_t)b * N + i) * Hq + h) * D;
+                for (int d = 0; d < D; ++d) qd[d] = bf16_to_f64(qi[d]);
+                for (int j = 0; j < S; ++j) allowed[j] = 1;
+                for (int t = 0; t < N; ++t) allowed[S + t] = (unsigned char)((mrow[t / 64] >> (t % 64)) & 1);
+                double m = -INFINITY;
+                for (int j = 0; j < S + N; ++j) {
+                    if (!allowed[j]) continue;
+                    double acc = 0.0;
+                    for (int d = 0; d < D; ++d) acc += qd[d] * bf16_to_f64(Kh[(size_t)j * D + d]);
+                    s[j] = scale * acc;
+                    if (s[j] > m) m = s[j];
+                }
+                double denom = 0.0;
+                for (int d = 0; d < D; ++d) o[d] = 0.0;
+                for (int j = 0; j < S + N; ++j) {
+                    if (!allowed[j]) continue;
+                    double w = exp(s[j] - m);
+                    denom += w;
+                    for (int d = 0; d < D; ++d) o[d] += w * bf16_to_f64(Vh[(size_t)j * D + d]);
+                }
+                if (denom > 0.0) {
+                    for (int d = 0; d < D; ++d) o[d] /= denom;
+                } else {
+                    for (int d = 0; d < D; ++d) o[d] = 0.0;
+                }
+                if (lse) lse[((size_t)b * Hq + h) * N + i] = denom > 0.0 ? m + log(denom) : -INFINITY;
+            }
+            free(s); free(allowed); free(qd);
+        }
+    }
+    return status;
+}
+
+/* Greedy (temperature 0) acceptance on a tree.  A non-root node a is "matched" iff
+ * draft_ids[a] == target_ids[parents[a]] (the target's greedy token after the parent is the drafted
+ * token).  Node i is accepted-reachable iff every non-root node on the chain i -> root is matched.
+ * The accepted path ends at the reachable node of greatest depth (smallest index among equals);
+ * path lists that chain from the root down; accept_len counts its nodes (root included);
+ * bonus = target_ids[last node of the path] (the token the target emits after the path). */
+int oracle_accept(const int32_t* draft_ids, const int32_t* target_ids, const int32_t* parents,
+                  int B, int N, int32_t* path, int32_t* accept_len, int32_t* bonus) {
+    for (int b = 0; b < B; ++b) {
+        const int32_t* par = parents + (size_t)b * N;
+        const int32_t* dr = draft_ids + (size_t)b * N;
+        const int32_t* tg = target_ids + (size_t)b * N;
+        int best = 0, best_depth = 0;
+        for (int i = 0; i < N; ++i) {
+            int ok = 1, d = 0;
+            for (int a = i; a != 0; a = par[a]) {
+                if (par[a] < 0 || par[a] >= a) return -1;
+                if (dr[a] != tg[par[a]]) ok = 0;
+                ++d;
+            }
+            if (ok && d > best_depth) { best = i; best_depth = d; }
+        }
+        int32_t* p = path + (size_t)b * N;
+        for (int k = 0; k < N; ++k) p[k] = -1;
+        int k = best_depth;
+        for (int a = best; ; a = par[a]) { p[k--] = a; if (a == 0) break; }
+        accept_len[b] = best_depth + 1;
+        bonus[b] = tg[best];
+    }
+    return 0;
+}
+
+/* KV commit for one layer's cache pair: for every sequence and kv head the rows at slots
+ * S + path[k], k < accept_len, are gathered into a temporary and then written to slots S + k
+ * (K and V alike).  Every other slot keeps its bytes.  kv_len_out[b] = S + accept_len (may be NULL). */
+int oracle_kv_compact(uint16_t* k_cache, uint16_t* v_cache, const int32_t* path,
+                      const int32_t* accept_len, const int32_t* kv_len, int32_t* kv_len_out,
+                      int B, int N, int Hkv, int D, int S_max) {
+    for (int b = 0; b < B; ++b) {
+        int S = kv_len[b], L = accept_len[b];
+        if (L < 1 || L > N || S < 0 || S + N > S_max) return -1;
+        for (int k = 0; k < L; ++k) {
+            int src = path[(size_t)b * N + k];
+            if (src < 0 || src >= N) return -2;
+        }
+        uint16_t* tmp = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)L * D);
+        if (!tmp) return -3;
+        for (int which = 0; which < 2; ++which) {
+            uint16_t* cache = which ? v_cache : k_cache;
+            for (int h = 0; h < Hkv; ++h) {
+                uint16_t* base = cache + ((size_t)b * Hkv + h) * (size_t)S_max * D;
+                for (int k = 0; k < L; ++k)
+                    memcpy(tmp + (size_t)k * D, base + (size_t)(S + path[(size_t)b * N + k]) * D,
+                           sizeof(uint16_t) * D);
+                for (int k = 0; k < L; ++k)
+                    memcpy(base + (size_t)(S + k) * D, tmp + (size_t)k * D, sizeof(uint16_t) * D);
+            }
+        }
+        free(tmp);
+        if (kv_len_out) kv_len_out[b] = S + L;
+    }
+    return 0;
+}
