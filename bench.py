@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-tree verification step (one JSON line on stdout).
+
+A *step* is one pass of the whole hot path over one batch of synthetic input:
+    vispec_tree_mask_build -> vispec_tree_verify_attn x L layers (each layer its own cache buffers)
+    -> vispec_accept -> vispec_kv_compact over all L layers.
+`value` is verify-attention KV GB/s: the K and V bytes the L attention calls must read
+(sum_b 2*(S_b+N)*Hkv*D*2 per layer) divided by the whole step's device time.  Inputs are resident in
+HBM before the timed region; the L layers' caches total far more than L2, so no flush is needed.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config llava7b] [--impl reference]
+
+With N > 1 (torchrun, one rank per GPU) every rank runs an independent replica of the workload: the
+path has no exchange step, so there is no collective on the data path; `value` sums the replicas.
+`--impl reference` times the CPU fp64 oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verify-attention KV GB/s (tree-verify step: mask + L x attention + accept + compact)"
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) of one attention launch of the benchmarked workload, from the ncu
+# capture summarised under profiles/; None until a capture exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="llava7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+            self.out.close()
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+            sm = [float(r[0]) for r in rows if len(r) >= 7]
+            power = [float(r[2]) for r in rows if len(r) >= 7]
+            if sm:
+                busy = [s for s, p in zip(sm, power) if p >= 0.5 * max(power)] or sm
+                res["sm_mhz"] = float(np.median(busy))
+                res["sm_max_mhz"] = float(rows[0][1])
+                res["power_w_max"] = max(power)
+                res["samples"] = len(sm)
+                names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+                for j, n in enumerate(names):
+                    if any(r[3 + j].strip().lower().startswith("active") for r in rows if len(r) >= 7):
+                        res["reasons"].append(n)
+        except Exception:
+            pass
+        return res
+
+
+# ------------------------------------------------------------------------------------ workload
+
+def build_host_inputs(cfg, layers):
+    """Seeded host inputs for all layers (numpy, bf16 bit patterns); generation is threaded."""
+    from paper_2509_15235_b200 import synth
+    tree = synth.make_tree_inputs(cfg)
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        per_layer = list(ex.map(lambda l: synth.make_layer_tensors(cfg, l), range(layers)))
+    return tree, per_layer
+
+
+class DeviceWorkload:
+    """All device buffers of one replica plus the step function that drives the C ABI."""
+
+    def __init__(self, cfg, tree, per_layer, device):
+        import torch
+        from paper_2509_15235_b200 import binding
+        self.torch, self.cfg = torch, cfg
+        self.L = len(per_layer)
+        dev = torch.device("cuda", device)
+        self.dev = dev
+        B, N, Hq, Hkv, D = cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D
+        self.ctx = binding.VerifyContext(B, N, Hq, Hkv, D, cfg.S_max, self.L, device=device)
+
+        def bf16(bits):
+            return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+        def i32(a):
+            return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+
+        self.k = [bf16(x["k_cache"]) for x in per_layer]
+        self.v = [bf16(x["v_cache"]) for x in per_layer]
+        self.q = torch.stack([bf16(x["q"]) for x in per_layer])            # [L,B,N,Hq,D]
+        self.out = torch.zeros_like(self.q)
+        for l in range(self.L):
+            self.ctx.cache_register(l, self.k[l], self.v[l])
+        self.parents, self.draft, self.target = i32(tree["parents"]), i32(tree["draft_ids"]), i32(tree["target_ids"])
+        self.kv_len = i32(tree["kv_len"])
+        W = (N + 63) // 64
+        self.mask = torch.zeros((B, N, W), dtype=torch.int64, device=dev)
+        self.depth = torch.zeros((B, N), dtype=torch.int32, device=dev)
+        self.path = torch.zeros((B, N), dtype=torch.int32, device=dev)
+        self.alen = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.bonus = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.new_len = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.scale = 1.0 / math.sqrt(D)
+        self.kv_bytes_per_layer = cfg.kv_bytes_per_layer(tree["kv_len"])
+
+    def step(self, ev_attn=None):
+        c = self.ctx
+        c.tree_mask_build(self.parents, self.mask, self.depth)
+        if ev_attn:
+            ev_attn[0].record()
+        for l in range(self.L):
+            c.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
+        if ev_attn:
+            ev_attn[1].record()
+        c.accept(self.draft, self.target, self.parents, self.path, self.alen, self.bonus)
+        # kv_len itself is left as it was so that every step sees the same workload
+        c.kv_compact(0, self.L, self.path, self.alen, self.kv_len, self.new_len)
+
+
+class HostStep:
+    """End-to-end step: the cycle's inputs start in pinned host memory and its results end there.
+    Per step: H2D of parents / draft_ids / target_ids / kv_len, of q for all layers and of the tree's
+    new K/V rows for all layers (written to slots S..S+N-1 of the resident caches); D2H of the
+    attention output of all layers, the accepted path, accept_len, bonus and the new kv_len.
+    The committed prefix of the cache is state that lives on the device across cycles."""
+
+    def __init__(self, wl: DeviceWorkload, tree, per_layer):
+        torch = wl.torch
+        self.wl = wl
+        cfg = wl.cfg
+        pin = lambda t: t.pin_memory()
+        self.h_q = pin(wl.q.cpu())
+        self.h_out = pin(torch.zeros_like(self.h_q))
+        S = tree["kv_len"]
+        N = cfg.N
+        # new rows [L,B,Hkv,N,D] gathered from the synthetic caches (host side, outside the timed region)
+        rows_k = np.stack([np.stack([x["k_cache"][b, :, S[b]:S[b] + N] for b in range(cfg.B)]) for x in per_layer])
+        rows_v = np.stack([np.stack([x["v_cache"][b, :, S[b]:S[b] + N] for b in range(cfg.B)]) for x in per_layer])
+        self.h_newk = pin(torch.from_numpy(rows_k.view(np.int16)).view(torch.bfloat16))
+        self.h_newv = pin(torch.from_numpy(rows_v.view(np.int16)).view(torch.bfloat16))
+        self.d_newk = torch.empty_like(self.h_newk, device=wl.dev)
+        self.d_newv = torch.empty_like(self.h_newv, device=wl.dev)
+        self.h_ints = pin(torch.from_numpy(np.concatenate([tree["parents"].ravel(), tree["draft_ids"].ravel(),
+                                                           tree["target_ids"].ravel(), tree["kv_len"].ravel()]).astype(np.int32)))
+        self.d_ints = torch.empty_like(self.h_ints, device=wl.dev)
+        BN = cfg.B * N
+        self.views = (self.d_ints[:BN].view(cfg.B, N), self.d_ints[BN:2 * BN].view(cfg.B, N),
+                      self.d_ints[2 * BN:3 * BN].view(cfg.B, N), self.d_ints[3 * BN:])
+        self.d_res = torch.zeros(BN + 3 * cfg.B, dtype=torch.int32, device=wl.dev)
+        self.h_res = pin(torch.zeros(BN + 3 * cfg.B, dtype=torch.int32))
+        self.S = [int(s) for s in S]
+        self.h2d = (self.h_q.numel() + self.h_newk.numel() + self.h_newv.numel()) * 2 + self.h_ints.numel() * 4
+        self.d2h = self.h_out.numel() * 2 + self.h_res.numel() * 4
+
+    def step(self):
+        wl, cfg = self.wl, self.wl.cfg
+        torch = wl.torch
+        B, N = cfg.B, cfg.N
+        self.d_ints.copy_(self.h_ints, non_blocking=True)
+        wl.q.copy_(self.h_q, non_blocking=True)
+        self.d_newk.copy_(self.h_newk, non_blocking=True)
+        self.d_newv.copy_(self.h_newv, non_blocking=True)
+        parents, draft, target, kv_len = self.views
+        for l in range(wl.L):                      # place the tree's rows behind the committed prefix
+            for b in range(B):
+                s = self.S[b]
+                wl.k[l][b, :, s:s + N].copy_(self.d_newk[l, b], non_blocking=True)
+                wl.v[l][b, :, s:s + N].copy_(self.d_newv[l, b], non_blocking=True)
+        c = wl.ctx
+        path = self.d_res[:B * N].view(B, N)
+        alen, bonus, new_len = self.d_res[B * N:B * N + B], self.d_res[B * N + B:B * N + 2 * B], self.d_res[B * N + 2 * B:]
+        c.tree_mask_build(parents, wl.mask, wl.depth)
+        for l in range(wl.L):
+            c.tree_verify_attn(l, wl.q[l], kv_len, wl.mask, wl.scale, wl.out[l])
+        c.accept(draft, target, parents, path, alen, bonus)
+        c.kv_compact(0, wl.L, path, alen, kv_len, new_len)
+        self.h_out.copy_(wl.out, non_blocking=True)
+        self.h_res.copy_(self.d_res, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller reads accept_len to go on
+
+
+# ------------------------------------------------------------------------------------ oracle legs
+
+def oracle_sample(cfg, tree, layer0, budget_heads):
+    """Time the oracle, as it stands, on one layer restricted to `budget_heads` kv heads (all of
+    their query heads, all nodes, the full cache length) plus mask, acceptance and commit."""
+    import oracle
+    G = cfg.G
+    hk = min(cfg.Hkv, budget_heads)
+    q = layer0["q"][:, :, :hk * G]
+    k = layer0["k_cache"][:, :hk]
+    v = layer0["v_cache"][:, :hk]
+    t0 = time.perf_counter()
+    mask, _, _ = oracle.tree_mask(tree["parents"])
+    oracle.tree_attn(q, k, v, tree["kv_len"], mask, 1.0 / math.sqrt(cfg.D), want_lse=False)
+    path, alen, _ = oracle.accept(tree["draft_ids"], tree["target_ids"], tree["parents"])
+    oracle.kv_compact(k, v, path, alen, tree["kv_len"])
+    dt = time.perf_counter() - t0
+    kv_bytes = int(sum(2 * (int(s) + cfg.N) * hk * cfg.D * 2 for s in tree["kv_len"]))
+    return kv_bytes / dt / 1e9, dt, hk, oracle.num_threads()
+
+
+def run_reference(args):
+    """The reference arm is the CPU oracle timed on the host cores (there is no reference code)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2509_15235_b200 import synth
+    cfg = synth.get_config(args.config)
+    tree = synth.make_tree_inputs(cfg)
+    layer0 = synth.make_layer_tensors(cfg, 0)
+    heads = min(cfg.Hkv, 8)
+    for _ in range(args.warmup):
+        oracle_sample(cfg, tree, layer0, heads)
+    t0 = time.perf_counter()
+    vals = [oracle_sample(cfg, tree, layer0, heads) for _ in range(args.steps)]
+    total = time.perf_counter() - t0
+    gbs = float(np.mean([v[0] for v in vals]))
+    sample = (f"per step: 1 of {cfg.layers} layers, {vals[0][2]} of {cfg.Hkv} kv heads, all nodes, full KV length, "
+              f"plus mask/accept/commit; fp64 C + OpenMP")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "note": "CPU oracle on host cores; bounded sample of the workload"},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": vals[0][3], "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------ main arm
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    from paper_2509_15235_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    cfg = synth.get_config(args.config)
+    warmup = max(args.warmup, 3)
+
+    tree, per_layer = build_host_inputs(cfg, cfg.layers)
+    wl = DeviceWorkload(cfg, tree, per_layer, local)
+    L = wl.L
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    for _ in range(warmup):
+        wl.step()
+    barrier()
+    assert wl.ctx.status_poll() == 0
+    launches0 = wl.ctx.launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for s in range(args.steps):
+        wl.step(evs[s])
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    attn_ms = sum(a.elapsed_time(b) for a, b in evs)
+    launches = wl.ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    status = wl.ctx.status_poll()
+
+    t = torch.tensor([ms_total, attn_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, attn_ms = float(t[0]), float(t[1])
+    kv_bytes_step = wl.kv_bytes_per_layer * L
+    value = world * kv_bytes_step * args.steps / (ms_total * 1e-3) / 1e9
+
+    # ---- end-to-end timing (host buffers in, host results out) ----
+    e2e = None
+    if not args.no_e2e:
+        hs = HostStep(wl, tree, per_layer)
+        for _ in range(3):
+            hs.step()
+        barrier()
+        n_e2e = max(3, min(args.steps, 10))
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            hs.step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * kv_bytes_step * n_e2e / float(tt[0]) / 1e9, "unit": "GB/s",
+               "h2d_bytes_per_step": hs.h2d, "d2h_bytes_per_step": hs.d2h, "steps": n_e2e,
+               "ms_per_step": 1e3 * float(tt[0]) / n_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    attn_s = attn_ms * 1e-3 / (args.steps * L)
+    achieved = wl.kv_bytes_per_layer / attn_s / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D, "N": cfg.N,
+                   "kv_len": [int(s) for s in tree["kv_len"]], "layers": L,
+                   "kv_bytes_per_layer": wl.kv_bytes_per_layer,
+                   "l2": f"inputs larger than L2: {L} layers x {wl.kv_bytes_per_layer / 1e6:.1f} MB rotate, no flush",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
+        "attn_us_per_layer": attn_s * 1e6,
+        "pct_of_8TBs": 100.0 * achieved / 8000.0,
+        "status_word": status,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "kernel": "vispec_tree_verify_attn (main kernel + merge)",
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)},
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+    }
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline:
+        gbs, dt, hk, cores = oracle_sample(cfg, tree, per_layer[0], min(cfg.Hkv, 32))
+        line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                "sample": f"1 of {L} layers, {hk} of {cfg.Hkv} kv heads, all nodes, full KV length, plus "
+                                          f"mask/accept/commit ({dt:.2f} s of fp64 C + OpenMP)"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

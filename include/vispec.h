@@ -1,0 +1,164 @@
+/*
+ * vispec.h - C ABI of the draft-tree verification step of speculative decoding for
+ * vision-language models (ViSpec, arXiv 2509.15235), written for NVIDIA B200 (sm_100a).
+ *
+ * The paper's decoding loop (Sec. 3.1) alternates drafting and verification: the target model
+ * scores a whole tree of drafted tokens in one forward, keeps the longest root path whose tokens
+ * it would have produced itself, and commits that path to its pre-allocated KV cache (App. A).
+ * This library is the attention-side hot path of that verification:
+ *
+ *   vispec_tree_mask_build   parent array of the draft tree -> per-node ancestor bitmask
+ *   vispec_tree_verify_attn  tree-masked attention (Eq. 1 with scale) of all tree queries against
+ *                            the long, image-token dominated bf16 KV cache of one layer
+ *   vispec_accept            greedy (temperature 0) acceptance walk -> accepted path, bonus token
+ *   vispec_kv_compact        gather the accepted path's K/V rows into the contiguous cache
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".  The library never takes
+ *     ownership of caller memory and never frees it.
+ *   - Hot calls (mask, attention, accept, compact) allocate nothing, never synchronise with the
+ *     host and enqueue their work on `stream` (a cudaStream_t passed as void*; NULL = default).
+ *   - Every function returns VISPEC_OK (0) or a negative vispec_status.  Errors that only the
+ *     device can see (a bad parent index, kv_len + N beyond the allocation, a bounded wait that
+ *     ran out) are recorded in a device status word that vispec_status_poll reads; the kernel
+ *     that met the error skips the offending work instead of faulting.
+ *   - Notation: B sequences, N tree nodes INCLUDING the root (node 0, the last committed token's
+ *     successor; parents[b][0] = -1), W = ceil(N/64) mask words, Hq/Hkv query/KV heads,
+ *     G = Hq/Hkv, D head dim, S = kv_len[b] committed slots, S_max allocated slots, L layers.
+ *   - Layouts (row-major): q, out [B,N,Hq,D] bf16;  k_cache, v_cache [B,Hkv,S_max,D] bf16 per layer;
+ *     tree node i's K/V rows sit at slot S+i of its sequence when attention is called;
+ *     tree_mask [B,N,W] uint64 (bit t of row i: node t is visible to node i);
+ *     parents, draft_ids, target_ids, path [B,N] int32; kv_len, accept_len, bonus [B] int32.
+ */
+#ifndef VISPEC_H_
+#define VISPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum vispec_status {
+    VISPEC_OK = 0,
+    VISPEC_E_NULL = -1,         /* a required pointer is NULL */
+    VISPEC_E_ALIGN = -2,        /* a pointer misses its alignment (16 B tensors, 128 B caches) */
+    VISPEC_E_SHAPE = -3,        /* a size outside the supported set, or inconsistent with the context */
+    VISPEC_E_RANGE = -4,        /* an index (layer, device, kv_len + N) out of range */
+    VISPEC_E_UNSUPPORTED = -5,  /* valid request this build cannot serve */
+    VISPEC_E_CUDA = -6,         /* a CUDA runtime/driver call failed */
+    VISPEC_E_TIMEOUT = -7,      /* a bounded device-side wait gave up (status word only) */
+    VISPEC_E_BAD_TREE = -8,     /* parents[b][i] not in [0,i) for i>0, or parents[b][0] != -1 */
+    VISPEC_E_UNREGISTERED = -9, /* layer has no registered cache, or pointers differ from it */
+    VISPEC_E_WORKSPACE = -10    /* workspace missing or too small */
+} vispec_status;
+
+#define VISPEC_MAX_TREE_NODES 128
+
+typedef struct vispec_shape {
+    int32_t B_max;   /* most sequences per call */
+    int32_t N_max;   /* most tree nodes per sequence, 1..128 */
+    int32_t Hq;      /* query heads */
+    int32_t Hkv;     /* key/value heads, divides Hq */
+    int32_t D;       /* head dimension: 64 or 128 */
+    int32_t S_max;   /* allocated cache slots per (sequence, kv head) */
+    int32_t layers;  /* number of cache pairs that may be registered */
+} vispec_shape;
+
+typedef struct vispec_ctx vispec_ctx;  /* opaque; owns only descriptors and a device status word */
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* vispec_strerror(int status);
+
+/* Create a context for one model shape on CUDA device `device`.  Not a hot call: it allocates a few
+ * hundred bytes of device memory (status word, per-layer pointer table).  `*out` (host) receives the
+ * context.  Errors: E_NULL, E_SHAPE (D not 64/128, Hq % Hkv != 0, N_max > 128, a non-positive size),
+ * E_RANGE (no such device), E_CUDA. */
+int vispec_ctx_create(vispec_ctx** out, const vispec_shape* shape /*host*/, int device);
+
+/* Destroy a context and the small device allocations it made.  Caller memory (caches, workspace)
+ * is untouched.  NULL is accepted. */
+int vispec_ctx_destroy(vispec_ctx* ctx);
+
+/* Bytes of scratch the attention needs for `shape` on the context's device: split-KV partial
+ * results (fp32) plus arrival counters.  `*out` is host memory. */
+int vispec_workspace_bytes(const vispec_ctx* ctx, size_t* out /*host*/);
+
+/* Hand the context a caller-owned device buffer of at least vispec_workspace_bytes() bytes, 256-byte
+ * aligned.  The library zeroes its counters once here (enqueued on the default stream and
+ * synchronised: not a hot call).  The buffer must stay alive and must not be shared by calls that
+ * overlap on the GPU.  Errors: E_NULL, E_ALIGN, E_WORKSPACE (too small), E_CUDA. */
+int vispec_ctx_set_workspace(vispec_ctx* ctx, void* workspace, size_t bytes);
+
+/* Register layer `layer`'s cache pair [B_max,Hkv,S_max,D] bf16 (App. A: pre-allocated KV cache).
+ * Builds the TMA tensor maps for these base pointers and records them for vispec_kv_compact; call
+ * again if the allocator moves a cache.  Pointers must be 128-byte aligned.  Not a hot call (one
+ * small host->device copy).  Errors: E_NULL, E_ALIGN, E_RANGE (layer), E_CUDA. */
+int vispec_cache_register(vispec_ctx* ctx, int layer, void* k_cache, void* v_cache);
+
+/* Ancestor mask of a draft tree (the tree of Sec. 3.1 / App. A, given as a parent array):
+ *   tree_mask[b][i] = { i } U tree_mask[b][parents[b][i]],  depth[b][i] = |tree_mask[b][i]| - 1.
+ * parents [B,N] int32 with parents[b][0] = -1 and 0 <= parents[b][i] < i.  A node whose chain
+ * to the root meets an invalid link (or parents[b][0] != -1) gets a row with its own bit only and
+ * depth 0, and the status word becomes VISPEC_E_BAD_TREE; nothing faults.  depth may be NULL.
+ * Host errors: E_NULL, E_SHAPE (B < 0, B > B_max, N < 1, N > N_max). */
+int vispec_tree_mask_build(vispec_ctx* ctx, const int32_t* parents, int B, int N,
+                           uint64_t* tree_mask, int32_t* depth, void* stream);
+
+/* Tree-masked attention of one layer (Eq. 1 of the paper, with the 1/sqrt(d) scale it omits given
+ * explicitly as `scale`).  For sequence b, query head h, node i:
+ *   allowed keys A = { j < S } U { S + t : bit t of tree_mask[b][i] },   S = kv_len[b]
+ *   out[b][i][h] = sum_{j in A} softmax_j(scale * <q[b][i][h], k[b][h/G][j]>) * v[b][h/G][j]
+ * computed with fp32 accumulation from bf16 inputs, rounded once to bf16 (nearest even).
+ * lse [B,Hq,N] fp32 (optional, may be NULL) receives log sum_{j in A} exp(score_j).
+ * An empty A gives out = 0 and lse = -inf.  tree_mask is an INPUT (any bit pattern is honoured,
+ * it is never re-derived from parents).  Cache slots at or beyond S + N are never interpreted
+ * (they may hold NaN patterns); tree rows that a node's mask hides get weight exactly 0 and must
+ * hold finite values, as rows written by the K/V projection do.  `positions` [B,N] (kv_len + depth) is accepted for interface
+ * completeness; q and the cached k arrive already rotated, so it is not read.  It may be NULL.
+ * k_cache / v_cache must be the pointers registered for `layer` (or NULL to use them).
+ * A sequence with kv_len[b] < 0 or kv_len[b] + N > S_max gets out = 0 and the status word
+ * VISPEC_E_RANGE.  Needs a workspace (vispec_ctx_set_workspace).
+ * Host errors: E_NULL, E_ALIGN (q/out 16 B), E_SHAPE, E_RANGE (layer), E_UNREGISTERED, E_WORKSPACE. */
+int vispec_tree_verify_attn(vispec_ctx* ctx, int layer, const void* q, const void* k_cache,
+                            const void* v_cache, const int32_t* kv_len, const uint64_t* tree_mask,
+                            const int32_t* positions, int B, int N, float scale, void* out,
+                            float* lse, void* stream);
+
+/* Greedy acceptance (Sec. 3.1 at temperature 0; Table 1 upper half).  target_ids[b][i] is the
+ * target model's greedy token after node i; non-root node a is matched iff
+ * draft_ids[b][a] == target_ids[b][parents[b][a]]; the accepted path ends at the deepest node whose
+ * whole chain to the root is matched (smallest index among equally deep ones).
+ *   path[b][0..accept_len) = that chain from the root (always node 0) downward, rest padded with -1
+ *   accept_len[b] >= 1 counts its nodes; tau of Sec. 5.1 is accept_len - 1
+ *   bonus[b] = target_ids[b][last path node], the next cycle's root token
+ * draft_ids[b][0] is ignored.  Invalid parents: that sequence returns the root only and the status
+ * word VISPEC_E_BAD_TREE.  Host errors: E_NULL, E_SHAPE. */
+int vispec_accept(vispec_ctx* ctx, const int32_t* draft_ids, const int32_t* target_ids,
+                  const int32_t* parents, int B, int N, int32_t* path, int32_t* accept_len,
+                  int32_t* bonus, void* stream);
+
+/* Commit (App. A): for every registered layer in [layer_begin, layer_end), sequence and kv head, the
+ * rows at slots S + path[b][k], k < accept_len[b], are gathered and then written to slots S + k, for
+ * K and V, in place (gather-then-scatter: correct although a destination may be another entry's
+ * source).  All other slots keep their bytes.  kv_len_out[b] = S + accept_len[b] (may be NULL; must
+ * NOT alias kv_len, which other thread blocks of the same launch still read: E_SHAPE).  `N` is the row
+ * length of `path`; a valid path is strictly increasing with path[b][k] >= k.  A sequence whose accept_len, path entry or
+ * kv_len is out of range is skipped with status word VISPEC_E_RANGE.
+ * Host errors: E_NULL, E_SHAPE, E_RANGE (layers), E_UNREGISTERED. */
+int vispec_kv_compact(vispec_ctx* ctx, int layer_begin, int layer_end, const int32_t* path,
+                      const int32_t* accept_len, const int32_t* kv_len, int32_t* kv_len_out,
+                      int B, int N, void* stream);
+
+/* Read and clear the device status word (synchronises `stream`; not a hot call).
+ * `*code` (host) receives VISPEC_OK or the first asynchronous error recorded since the last poll. */
+int vispec_status_poll(vispec_ctx* ctx, int* code /*host*/, void* stream);
+
+/* Number of kernels the library has launched through this context since creation (host counter). */
+int vispec_launch_count(const vispec_ctx* ctx, uint64_t* out /*host*/);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VISPEC_H_ */

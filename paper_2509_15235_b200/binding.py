@@ -1,0 +1,175 @@
+"""Thin ctypes binding of libvispec.so: argument marshalling only.
+
+Every step of the verification path runs in the library's CUDA kernels; torch is used here for
+device memory and streams.  There is no CPU fallback: if the shared object is missing or CUDA is
+unavailable the import of the library (``load()``) raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvispec.so")
+
+VISPEC_OK = 0
+STATUS_NAMES = {
+    0: "VISPEC_OK", -1: "VISPEC_E_NULL", -2: "VISPEC_E_ALIGN", -3: "VISPEC_E_SHAPE", -4: "VISPEC_E_RANGE",
+    -5: "VISPEC_E_UNSUPPORTED", -6: "VISPEC_E_CUDA", -7: "VISPEC_E_TIMEOUT", -8: "VISPEC_E_BAD_TREE",
+    -9: "VISPEC_E_UNREGISTERED", -10: "VISPEC_E_WORKSPACE",
+}
+EXPORTS = [
+    "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
+    "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
+    "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
+    "vispec_launch_count",
+]
+
+
+class VispecShape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("B_max", "N_max", "Hq", "Hkv", "D", "S_max", "layers")]
+
+
+class VispecError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)} ({strerror(code)})")
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load() -> ctypes.CDLL:
+    """dlopen the in-tree library.  Fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2509_15235_b200.build` "
+                              "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+        lib.vispec_strerror.restype = ctypes.c_char_p
+        lib.vispec_strerror.argtypes = [ci]
+        sigs = {
+            "vispec_ctx_create": [ctypes.POINTER(vp), ctypes.POINTER(VispecShape), ci],
+            "vispec_ctx_destroy": [vp],
+            "vispec_workspace_bytes": [vp, ctypes.POINTER(ctypes.c_size_t)],
+            "vispec_ctx_set_workspace": [vp, vp, ctypes.c_size_t],
+            "vispec_cache_register": [vp, ci, vp, vp],
+            "vispec_tree_mask_build": [vp, vp, ci, ci, vp, vp, vp],
+            "vispec_tree_verify_attn": [vp, ci, vp, vp, vp, vp, vp, vp, ci, ci, cf, vp, vp, vp],
+            "vispec_accept": [vp, vp, vp, vp, ci, ci, vp, vp, vp, vp],
+            "vispec_kv_compact": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp],
+            "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
+            "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
+        }
+        for name, argtypes in sigs.items():
+            fn = getattr(lib, name)
+            fn.restype = ci
+            fn.argtypes = argtypes
+        _lib = lib
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return load().vispec_strerror(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device pointers must come from contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code: int, where: str) -> None:
+    if code != VISPEC_OK:
+        raise VispecError(code, where)
+
+
+class VerifyContext:
+    """Owns a ``vispec_ctx`` plus the torch-allocated workspace it points at.
+
+    Method names mirror the C entry points; each is one C call on torch's current stream.
+    """
+
+    def __init__(self, B_max: int, N_max: int, Hq: int, Hkv: int, D: int, S_max: int, layers: int,
+                 device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libvispec needs a CUDA device (no CPU fallback exists)")
+        self.lib = load()
+        self.shape = VispecShape(B_max, N_max, Hq, Hkv, D, S_max, layers)
+        self.device = torch.device("cuda", device)
+        h = ctypes.c_void_p()
+        _check(self.lib.vispec_ctx_create(ctypes.byref(h), ctypes.byref(self.shape), device), "vispec_ctx_create")
+        self.handle = h
+        n = ctypes.c_size_t()
+        _check(self.lib.vispec_workspace_bytes(self.handle, ctypes.byref(n)), "vispec_workspace_bytes")
+        self.workspace = torch.empty(n.value, dtype=torch.uint8, device=self.device)
+        _check(self.lib.vispec_ctx_set_workspace(self.handle, _ptr(self.workspace), n.value),
+               "vispec_ctx_set_workspace")
+        self._caches = {}
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            self.lib.vispec_ctx_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- registration ---------------------------------------------------------------------------
+    def cache_register(self, layer: int, k_cache: torch.Tensor, v_cache: torch.Tensor) -> None:
+        _check(self.lib.vispec_cache_register(self.handle, layer, _ptr(k_cache), _ptr(v_cache)),
+               "vispec_cache_register")
+        self._caches[layer] = (k_cache, v_cache)   # keep the tensors alive
+
+    # -- hot calls --------------------------------------------------------------------------------
+    def tree_mask_build(self, parents: torch.Tensor, tree_mask: torch.Tensor,
+                        depth: Optional[torch.Tensor] = None) -> None:
+        B, N = parents.shape
+        _check(self.lib.vispec_tree_mask_build(self.handle, _ptr(parents), B, N, _ptr(tree_mask), _ptr(depth),
+                                               _stream()), "vispec_tree_mask_build")
+
+    def tree_verify_attn(self, layer: int, q: torch.Tensor, kv_len: torch.Tensor, tree_mask: torch.Tensor,
+                         scale: float, out: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                         positions: Optional[torch.Tensor] = None, k_cache: Optional[torch.Tensor] = None,
+                         v_cache: Optional[torch.Tensor] = None) -> None:
+        B, N = q.shape[0], q.shape[1]
+        _check(self.lib.vispec_tree_verify_attn(self.handle, layer, _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                                _ptr(kv_len), _ptr(tree_mask), _ptr(positions), B, N,
+                                                ctypes.c_float(scale), _ptr(out), _ptr(lse), _stream()),
+               "vispec_tree_verify_attn")
+
+    def accept(self, draft_ids: torch.Tensor, target_ids: torch.Tensor, parents: torch.Tensor,
+               path: torch.Tensor, accept_len: torch.Tensor, bonus: torch.Tensor) -> None:
+        B, N = parents.shape
+        _check(self.lib.vispec_accept(self.handle, _ptr(draft_ids), _ptr(target_ids), _ptr(parents), B, N,
+                                      _ptr(path), _ptr(accept_len), _ptr(bonus), _stream()), "vispec_accept")
+
+    def kv_compact(self, layer_begin: int, layer_end: int, path: torch.Tensor, accept_len: torch.Tensor,
+                   kv_len: torch.Tensor, kv_len_out: Optional[torch.Tensor] = None) -> None:
+        B, N = path.shape
+        _check(self.lib.vispec_kv_compact(self.handle, layer_begin, layer_end, _ptr(path), _ptr(accept_len),
+                                          _ptr(kv_len), _ptr(kv_len_out), B, N, _stream()), "vispec_kv_compact")
+
+    # -- diagnostics ------------------------------------------------------------------------------
+    def status_poll(self) -> int:
+        code = ctypes.c_int()
+        _check(self.lib.vispec_status_poll(self.handle, ctypes.byref(code), _stream()), "vispec_status_poll")
+        return code.value
+
+    def launch_count(self) -> int:
+        n = ctypes.c_uint64()
+        _check(self.lib.vispec_launch_count(self.handle, ctypes.byref(n)), "vispec_launch_count")
+        return n.value

@@ -1,0 +1,190 @@
+// Integer kernels of the verification step: ancestor mask, greedy acceptance, KV commit.
+// All three are latency-bound (a few KB of traffic); each is a single launch.
+#include "vispec_internal.h"
+
+namespace vispec {
+
+__device__ __forceinline__ void record_status(int* status, int code) {
+    if (status) atomicCAS(status, 0, code);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Ancestor mask (tree of Sec. 3.1 / App. A).  One block per sequence, one thread per node: the
+// thread follows its node's parent links and ORs the visited indices into a 128-bit set.
+// A chain that meets an invalid link yields the self bit only and flags VISPEC_E_BAD_TREE.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+tree_mask_kernel(const int32_t* __restrict__ parents, int N, uint64_t* __restrict__ mask,
+                 int32_t* __restrict__ depth, int* status) {
+    __shared__ int32_t par[VISPEC_MAX_TREE_NODES];
+    const int b = blockIdx.x, i = threadIdx.x;
+    if (i < N) par[i] = parents[(size_t)b * N + i];
+    __syncthreads();
+    if (i >= N) return;
+    const int W = (N + 63) >> 6;
+    uint64_t m0 = 0, m1 = 0;
+    bool ok = (par[0] == -1);
+    int a = i, d = 0;
+    while (ok) {
+        if (a < 64) m0 |= 1ull << a; else m1 |= 1ull << (a - 64);
+        if (a == 0) break;
+        const int p = par[a];
+        if (p < 0 || p >= a) { ok = false; break; }
+        a = p;
+        ++d;
+    }
+    if (!ok) {
+        m0 = i < 64 ? 1ull << i : 0;
+        m1 = i < 64 ? 0 : 1ull << (i - 64);
+        d = 0;
+        record_status(status, VISPEC_E_BAD_TREE);
+    }
+    uint64_t* row = mask + ((size_t)b * N + i) * W;
+    row[0] = m0;
+    if (W > 1) row[1] = m1;
+    if (depth) depth[(size_t)b * N + i] = d;
+}
+
+cudaError_t launch_tree_mask(const int32_t* parents, int B, int N, uint64_t* mask, int32_t* depth,
+                             int* status, cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    tree_mask_kernel<<<B, 128, 0, st>>>(parents, N, mask, depth, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Greedy acceptance (Sec. 3.1 at temperature 0).  One warp per sequence; lane l owns nodes
+// l, l+32, l+64, l+96.  matched bits are gathered with ballots into a 128-bit set; a node is
+// reachable iff its ancestor set minus the matched set is empty; the winner is the deepest
+// reachable node (smallest index among equals), found with a shuffle max-reduction on the key
+// depth*256 + (255 - index).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32)
+accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ target,
+              const int32_t* __restrict__ parents, int N, int32_t* __restrict__ path,
+              int32_t* __restrict__ accept_len, int32_t* __restrict__ bonus, int* status) {
+    __shared__ int32_t par[VISPEC_MAX_TREE_NODES];
+    __shared__ int32_t tgt[VISPEC_MAX_TREE_NODES];
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const size_t base = (size_t)b * N;
+    for (int i = lane; i < N; i += 32) { par[i] = parents[base + i]; tgt[i] = target[base + i]; }
+    __syncwarp();
+    // validity of the whole tree (every link must point to an earlier node)
+    bool tree_ok = true;
+    for (int i = lane; i < N; i += 32) tree_ok &= (i == 0) ? (par[0] == -1) : (par[i] >= 0 && par[i] < i);
+    tree_ok = __all_sync(0xffffffffu, tree_ok);
+
+    uint32_t matched[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const int i = w * 32 + lane;
+        bool m = false;
+        if (tree_ok && i < N) m = (i == 0) || (draft[base + i] == tgt[par[i]]);
+        matched[w] = __ballot_sync(0xffffffffu, m);
+    }
+    int best_key = -1;
+    if (tree_ok) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const int i = w * 32 + lane;
+            if (i < N) {
+                uint32_t anc[4] = {0, 0, 0, 0};
+                int d = 0;
+                for (int a = i; ; a = par[a]) { anc[a >> 5] |= 1u << (a & 31); if (a == 0) break; ++d; }
+                const bool reach = ((anc[0] & ~matched[0]) | (anc[1] & ~matched[1]) |
+                                    (anc[2] & ~matched[2]) | (anc[3] & ~matched[3])) == 0;
+                if (reach) best_key = max(best_key, d * 256 + (255 - i));
+            }
+        }
+    } else {
+        if (lane == 0) { best_key = 255; record_status(status, VISPEC_E_BAD_TREE); }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) best_key = max(best_key, __shfl_xor_sync(0xffffffffu, best_key, off));
+    const int best_depth = best_key >> 8;
+    const int best = 255 - (best_key & 255);
+    for (int k = lane; k < N; k += 32) if (k > best_depth) path[base + k] = -1;
+    if (lane == 0) {
+        int a = best;
+        for (int k = best_depth; k >= 0; --k) { path[base + k] = a; a = (a == 0) ? 0 : par[a]; }
+        accept_len[b] = best_depth + 1;
+        bonus[b] = tgt[best];
+    }
+}
+
+cudaError_t launch_accept(const int32_t* draft, const int32_t* target, const int32_t* parents, int B,
+                          int N, int32_t* path, int32_t* accept_len, int32_t* bonus, int* status,
+                          cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    accept_kernel<<<B, 32, 0, st>>>(draft, target, parents, N, path, accept_len, bonus, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// KV commit (App. A, pre-allocated cache).  One block per (layer, sequence, kv head); rows are
+// D*2 contiguous bytes and move as 16-byte vectors.  Entries are processed in passes of 16 path
+// positions in increasing order: gather the pass into shared memory, barrier, scatter.  Because the
+// path is strictly increasing with path[k] >= k, a pass writes only slots below every later pass's
+// sources, so the result equals gather-everything-then-scatter.  Entries with path[k] == k are
+// already in place and are skipped.
+// ------------------------------------------------------------------------------------------------
+constexpr int kCompactRows = 16;
+
+__global__ void __launch_bounds__(256)
+kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const int32_t* __restrict__ path,
+                  const int32_t* __restrict__ accept_len, const int32_t* __restrict__ kv_len,
+                  int32_t* __restrict__ kv_len_out, int N, int Hkv, int D, int S_max, int* status) {
+    __shared__ uint4 stage[2][kCompactRows][16];   // up to 256 B per row (D = 128)
+    __shared__ int32_t src_row[kCompactRows];
+    const int layer = layer_begin + blockIdx.z, b = blockIdx.y, h = blockIdx.x;
+    const int S = kv_len[b], L = accept_len[b];
+    const bool ok = (L >= 1 && L <= N && S >= 0 && S + N <= S_max);
+    if (!ok) {
+        if (threadIdx.x == 0) record_status(status, VISPEC_E_RANGE);
+        return;   // kv_len_out[b] keeps its previous value for a rejected sequence
+    }
+    const int chunks = D / 8;                        // 16-byte vectors per row
+    const int tensor = threadIdx.x >> 7;             // 0: K, 1: V
+    const int r = (threadIdx.x & 127) >> 3;          // row of the pass, 0..15
+    const int c0 = threadIdx.x & 7;                  // this thread moves chunks c0 and c0 + 8
+    uint4* base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]) +
+                  ((size_t)b * Hkv + h) * (size_t)S_max * chunks;
+    bool bad = false;
+    for (int k0 = 0; k0 < L; k0 += kCompactRows) {
+        if (threadIdx.x < kCompactRows) {
+            const int k = k0 + threadIdx.x;
+            int s = (k < L) ? path[(size_t)b * N + k] : -1;
+            if (k < L && (s < k || s >= N)) { s = -1; bad = true; }
+            src_row[threadIdx.x] = (s == k) ? -1 : s;   // -1: nothing to move
+        }
+        __syncthreads();
+        const int s = src_row[r];
+        if (s >= 0) {
+            const uint4* src = base + (size_t)(S + s) * chunks;
+            if (c0 < chunks) stage[tensor][r][c0] = src[c0];
+            if (c0 + 8 < chunks) stage[tensor][r][c0 + 8] = src[c0 + 8];
+        }
+        __syncthreads();
+        if (s >= 0) {
+            uint4* dst = base + (size_t)(S + k0 + r) * chunks;
+            if (c0 < chunks) dst[c0] = stage[tensor][r][c0];
+            if (c0 + 8 < chunks) dst[c0 + 8] = stage[tensor][r][c0 + 8];
+        }
+        __syncthreads();
+    }
+    if (bad) record_status(status, VISPEC_E_RANGE);
+    if (kv_len_out && blockIdx.x == 0 && blockIdx.z == 0 && threadIdx.x == 0) kv_len_out[b] = S + L;
+}
+
+cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int layer_end,
+                              const int32_t* path, const int32_t* accept_len, const int32_t* kv_len,
+                              int32_t* kv_len_out, int B, int N, int Hkv, int D, int S_max, int* status,
+                              cudaStream_t st) {
+    if (B == 0 || layer_end <= layer_begin) return cudaSuccess;
+    dim3 grid(Hkv, B, layer_end - layer_begin);
+    kv_compact_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, path, accept_len, kv_len, kv_len_out,
+                                            N, Hkv, D, S_max, status);
+    return cudaGetLastError();
+}
+
+}  // namespace vispec

@@ -1,0 +1,230 @@
+// C ABI of libvispec: context management, argument validation, dispatch to the kernels.
+#include <cstring>
+#include <new>
+
+#include "vispec_internal.h"
+
+namespace vispec {
+
+size_t workspace_bytes(const vispec_shape& s, int sm_count) {
+    const int G = s.Hq / s.Hkv;
+    const size_t units64 = (size_t)s.B_max * s.Hkv * ((G * s.N_max + 63) / 64);
+    const size_t slot = slot_bytes(s.D);
+    // generic kernel: at most 4*SMs + units partials of 64 rows (half slots);
+    // persistent kernel: at most two partials of 128 rows per CTA, one CTA per SM.
+    return kCounterBytes + (4 * (size_t)sm_count + units64) * (slot / 2) + 2 * (size_t)sm_count * slot;
+}
+
+}  // namespace vispec
+
+using namespace vispec;
+
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* vispec_strerror(int status) {
+    switch (status) {
+        case VISPEC_OK: return "ok";
+        case VISPEC_E_NULL: return "required pointer is NULL";
+        case VISPEC_E_ALIGN: return "pointer is not sufficiently aligned";
+        case VISPEC_E_SHAPE: return "unsupported or inconsistent shape";
+        case VISPEC_E_RANGE: return "index or length out of range";
+        case VISPEC_E_UNSUPPORTED: return "request not supported by this build";
+        case VISPEC_E_CUDA: return "CUDA call failed";
+        case VISPEC_E_TIMEOUT: return "bounded device-side wait gave up";
+        case VISPEC_E_BAD_TREE: return "parent array is not a valid tree";
+        case VISPEC_E_UNREGISTERED: return "layer cache not registered (or pointers differ)";
+        case VISPEC_E_WORKSPACE: return "workspace missing or too small";
+        default: return "unknown status";
+    }
+}
+
+int vispec_ctx_create(vispec_ctx** out, const vispec_shape* s, int device) {
+    if (!out || !s) return VISPEC_E_NULL;
+    *out = nullptr;
+    if (s->B_max < 1 || s->N_max < 1 || s->N_max > VISPEC_MAX_TREE_NODES || s->Hq < 1 || s->Hkv < 1 ||
+        s->Hq % s->Hkv != 0 || (s->D != 64 && s->D != 128) || s->S_max < s->N_max || s->layers < 1)
+        return VISPEC_E_SHAPE;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess) return VISPEC_E_CUDA;
+    if (device < 0 || device >= n_dev) return VISPEC_E_RANGE;
+    if (cudaSetDevice(device) != cudaSuccess) return VISPEC_E_CUDA;
+    vispec_ctx* c = new (std::nothrow) vispec_ctx();
+    if (!c) return VISPEC_E_CUDA;
+    c->shape = *s;
+    c->device = device;
+    bool ok = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_cache_ptrs, sizeof(void*) * 2 * s->layers) == cudaSuccess;
+    ok = ok && cudaMemset(c->d_cache_ptrs, 0, sizeof(void*) * 2 * s->layers) == cudaSuccess;
+    ok = ok && init_attn_generic() == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) { vispec_ctx_destroy(c); return VISPEC_E_CUDA; }
+    c->h_k.assign(s->layers, nullptr);
+    c->h_v.assign(s->layers, nullptr);
+    c->k_map.resize(s->layers);
+    c->v_map.resize(s->layers);
+    *out = c;
+    return VISPEC_OK;
+}
+
+int vispec_ctx_destroy(vispec_ctx* c) {
+    if (!c) return VISPEC_OK;
+    if (c->d_status) cudaFree(c->d_status);
+    if (c->d_cache_ptrs) cudaFree(c->d_cache_ptrs);
+    delete c;
+    return VISPEC_OK;
+}
+
+int vispec_workspace_bytes(const vispec_ctx* c, size_t* out) {
+    if (!c || !out) return VISPEC_E_NULL;
+    *out = workspace_bytes(c->shape, c->sm_count);
+    return VISPEC_OK;
+}
+
+int vispec_ctx_set_workspace(vispec_ctx* c, void* ws, size_t bytes) {
+    if (!c || !ws) return VISPEC_E_NULL;
+    if (!aligned(ws, 256)) return VISPEC_E_ALIGN;
+    if (bytes < workspace_bytes(c->shape, c->sm_count)) return VISPEC_E_WORKSPACE;
+    if (cudaMemset(ws, 0, kCounterBytes) != cudaSuccess) return VISPEC_E_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return VISPEC_E_CUDA;
+    c->ws = ws;
+    c->ws_bytes = bytes;
+    return VISPEC_OK;
+}
+
+int vispec_cache_register(vispec_ctx* c, int layer, void* k_cache, void* v_cache) {
+    if (!c || !k_cache || !v_cache) return VISPEC_E_NULL;
+    if (layer < 0 || layer >= c->shape.layers) return VISPEC_E_RANGE;
+    if (!aligned(k_cache, 128) || !aligned(v_cache, 128)) return VISPEC_E_ALIGN;
+    const vispec_shape& s = c->shape;
+    if (s.D == 128) {
+        // 3-D view (d, slot, sequence*head) of a [B,Hkv,S_max,D] bf16 cache; one box = 64 d-columns
+        // (128 bytes, the swizzle span) x 64 slots.  Slots past S_max read as zero.
+        EncodeTiledFn enc = get_encode_fn();
+        if (!enc) return VISPEC_E_CUDA;
+        const cuuint64_t dims[3] = {(cuuint64_t)s.D, (cuuint64_t)s.S_max, (cuuint64_t)s.B_max * s.Hkv};
+        const cuuint64_t strides[2] = {(cuuint64_t)s.D * 2, (cuuint64_t)s.S_max * s.D * 2};
+        const cuuint32_t box[3] = {64, 64, 1};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        void* ptrs[2] = {k_cache, v_cache};
+        CUtensorMap* maps[2] = {&c->k_map[layer], &c->v_map[layer]};
+        for (int t = 0; t < 2; ++t) {
+            CUresult r = enc(maps[t], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ptrs[t], dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return VISPEC_E_CUDA;
+        }
+    }
+    void* pair[2] = {k_cache, v_cache};
+    if (cudaMemcpy(c->d_cache_ptrs + 2 * layer, pair, sizeof(pair), cudaMemcpyHostToDevice) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    c->h_k[layer] = k_cache;
+    c->h_v[layer] = v_cache;
+    return VISPEC_OK;
+}
+
+int vispec_tree_mask_build(vispec_ctx* c, const int32_t* parents, int B, int N, uint64_t* tree_mask,
+                           int32_t* depth, void* stream) {
+    if (!c || !parents || !tree_mask) return VISPEC_E_NULL;
+    if (B < 0 || B > c->shape.B_max || N < 1 || N > c->shape.N_max) return VISPEC_E_SHAPE;
+    if (launch_tree_mask(parents, B, N, tree_mask, depth, c->d_status, (cudaStream_t)stream) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
+int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void* k_cache, const void* v_cache,
+                            const int32_t* kv_len, const uint64_t* tree_mask, const int32_t* positions,
+                            int B, int N, float scale, void* out, float* lse, void* stream) {
+    (void)positions;
+    if (!c || !q || !kv_len || !tree_mask || !out) return VISPEC_E_NULL;
+    if (!aligned(q, 16) || !aligned(out, 16)) return VISPEC_E_ALIGN;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
+    if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
+    if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
+    if ((k_cache && k_cache != c->h_k[layer]) || (v_cache && v_cache != c->h_v[layer])) return VISPEC_E_UNREGISTERED;
+    if (!c->ws) return VISPEC_E_WORKSPACE;
+    AttnArgs a;
+    a.q = q; a.k = c->h_k[layer]; a.v = c->h_v[layer];
+    a.kv_len = kv_len; a.mask = tree_mask; a.out = out; a.lse = lse;
+    a.B = B; a.N = N; a.Hq = s.Hq; a.Hkv = s.Hkv; a.D = s.D; a.S_max = s.S_max;
+    a.scale = scale; a.ws = c->ws; a.ws_bytes = c->ws_bytes; a.status = c->d_status;
+    a.sm_count = c->sm_count;
+    a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
+    int n = 0;
+    cudaError_t err = launch_attn_generic(a, (cudaStream_t)stream, &n);
+    c->launches += n;
+    return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
+}
+
+int vispec_accept(vispec_ctx* c, const int32_t* draft_ids, const int32_t* target_ids, const int32_t* parents,
+                  int B, int N, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
+    if (!c || !draft_ids || !target_ids || !parents || !path || !accept_len || !bonus) return VISPEC_E_NULL;
+    if (B < 0 || B > c->shape.B_max || N < 1 || N > c->shape.N_max) return VISPEC_E_SHAPE;
+    if (launch_accept(draft_ids, target_ids, parents, B, N, path, accept_len, bonus, c->d_status,
+                      (cudaStream_t)stream) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
+int vispec_kv_compact(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* path,
+                      const int32_t* accept_len, const int32_t* kv_len, int32_t* kv_len_out, int B, int N,
+                      void* stream) {
+    if (!c || !path || !accept_len || !kv_len) return VISPEC_E_NULL;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
+    if (layer_begin < 0 || layer_end > s.layers || layer_begin > layer_end) return VISPEC_E_RANGE;
+    if (kv_len_out == kv_len) return VISPEC_E_SHAPE;
+    for (int l = layer_begin; l < layer_end; ++l)
+        if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
+    if (launch_kv_compact(c->d_cache_ptrs, layer_begin, layer_end, path, accept_len, kv_len, kv_len_out, B, N,
+                          s.Hkv, s.D, s.S_max, c->d_status, (cudaStream_t)stream) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0 && layer_end > layer_begin) c->launches += 1;
+    return VISPEC_OK;
+}
+
+int vispec_status_poll(vispec_ctx* c, int* code, void* stream) {
+    if (!c || !code) return VISPEC_E_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return VISPEC_E_CUDA;
+    if (cudaMemsetAsync(c->d_status, 0, sizeof(int), st) != cudaSuccess) return VISPEC_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return VISPEC_E_CUDA;
+    *code = v;
+    return VISPEC_OK;
+}
+
+int vispec_launch_count(const vispec_ctx* c, uint64_t* out) {
+    if (!c || !out) return VISPEC_E_NULL;
+    *out = c->launches;
+    return VISPEC_OK;
+}
+
+}  // extern "C"

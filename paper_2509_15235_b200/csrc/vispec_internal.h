@@ -1,0 +1,60 @@
+// Internal declarations shared by the translation units of libvispec (never installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <vector>
+
+#include "vispec.h"
+
+struct vispec_ctx {
+    vispec_shape shape;
+    int device = 0;
+    int sm_count = 0;
+    int* d_status = nullptr;        // device status word (first asynchronous error wins)
+    void** d_cache_ptrs = nullptr;  // device table [layers][2]: k_cache, v_cache
+    std::vector<void*> h_k, h_v;    // host copy of the registered pointers
+    std::vector<CUtensorMap> k_map, v_map;  // TMA descriptors per layer (D == 128 only)
+    void* ws = nullptr;             // caller-owned workspace
+    size_t ws_bytes = 0;
+    uint64_t launches = 0;
+};
+
+namespace vispec {
+
+// ---- workspace layout -------------------------------------------------------------------------
+// [0, kCounterBytes)            arrival counters (int32), zero between calls
+// [kCounterBytes, ...)          partial-result slots, each kSlotRows rows of (D fp32 + m + l)
+constexpr size_t kCounterBytes = 64 * 1024;
+constexpr int kSlotRows = 128;
+inline size_t slot_bytes(int D) { return (size_t)kSlotRows * ((size_t)D * 4 + 8); }
+size_t workspace_bytes(const vispec_shape& s, int sm_count);
+
+// ---- kernels' host launchers (each returns a cudaError_t from the launch) -----------------------
+cudaError_t launch_tree_mask(const int32_t* parents, int B, int N, uint64_t* mask, int32_t* depth,
+                             int* status, cudaStream_t st);
+cudaError_t launch_accept(const int32_t* draft, const int32_t* target, const int32_t* parents, int B,
+                          int N, int32_t* path, int32_t* accept_len, int32_t* bonus, int* status,
+                          cudaStream_t st);
+cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int layer_end,
+                              const int32_t* path, const int32_t* accept_len, const int32_t* kv_len,
+                              int32_t* kv_len_out, int B, int N, int Hkv, int D, int S_max, int* status,
+                              cudaStream_t st);
+
+struct AttnArgs {
+    const void* q; const void* k; const void* v;
+    const int32_t* kv_len; const uint64_t* mask;
+    void* out; float* lse;
+    int B, N, Hq, Hkv, D, S_max;
+    float scale;
+    void* ws; size_t ws_bytes;
+    int* status;
+    int sm_count;
+    const CUtensorMap* k_map; const CUtensorMap* v_map;
+};
+// Generic split-KV kernel on warp-level tensor-core instructions (any supported shape).
+cudaError_t init_attn_generic();   // once per device, with that device current
+cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, int* n_launches);
+
+}  // namespace vispec

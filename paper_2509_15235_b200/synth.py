@@ -101,8 +101,11 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """float32 -> bfloat16 bit patterns, round to nearest even (NaN kept quiet)."""
     x = np.ascontiguousarray(x, dtype=np.float32)
     u = x.view(np.uint32)
-    rounded = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
-    out = rounded.astype(np.uint16)
+    r = (u >> np.uint32(16)) & np.uint32(1)
+    r += np.uint32(0x7FFF)
+    r += u
+    r >>= np.uint32(16)
+    out = r.astype(np.uint16)
     nan = np.isnan(x)
     if nan.any():
         out[nan] = np.uint16(0x7FC0)
@@ -123,7 +126,7 @@ def tensor_seed(config_id: int, layer: int, tensor_id: int) -> int:
 
 
 def _rng(seed: int) -> np.random.Generator:
-    return np.random.Generator(np.random.Philox(int(seed)))
+    return np.random.Generator(np.random.SFC64(int(seed)))
 
 
 def normal_bf16(shape, seed: int) -> np.ndarray:
