@@ -126,6 +126,34 @@ int vispec_tree_verify_attn(vispec_ctx* ctx, int layer, const void* q, const voi
                             const int32_t* positions, int B, int N, float scale, void* out,
                             float* lse, void* stream);
 
+/* Attention without any allocation (the paper has no counterpart: this entry point exists for
+ * deployment, not for the method).  It is for callers that cannot obtain device memory when they
+ * need to run: a serving process whose memory pool is fixed at start-up, a plugin that receives
+ * tensors but no allocator, code on a latency-critical stream where cudaMalloc's implicit
+ * device synchronisation is not acceptable.  It computes exactly what vispec_tree_verify_attn
+ * computes, but needs no context, no registration and no workspace: the split-KV partial results go
+ * to a 16 MiB array that is part of the library image (static device memory, held on every GPU that
+ * loads the library until the process exits).  The function calls no cudaMalloc/cudaFree and no
+ * allocating library routine.
+ *   - Arguments as in vispec_tree_verify_attn, with the shape given explicitly (Hq, Hkv, D in
+ *     {64,128}, S_max) and the caches passed directly ([B,Hkv,S_max,D] bf16, 16-byte aligned).
+ *   - status_word: optional DEVICE int32 that receives VISPEC_E_RANGE (compare-and-swap from 0) if a
+ *     sequence has kv_len < 0 or kv_len + N > S_max (that sequence's output is zero); may be NULL.
+ *   - Limit: B * Hkv * ceil(G*N/64) partial-result units must fit the array with two KV splits,
+ *     i.e. 64 KiB + 2 * units * 64 * (4*D + 8) bytes <= 16 MiB (at D = 128: 251 units).  Beyond
+ *     that the call returns VISPEC_E_WORKSPACE and does nothing.
+ *   - The first call on each device looks up the array's device address and sets one kernel
+ *     attribute; make that first call outside any stream capture, with the device current.
+ *   - All calls share the one array, and it keeps the previous call's contents.  Nothing in it has
+ *     to start at zero (every partial is written before it is read), so no clearing is done; but two
+ *     calls that overlap on the GPU (different streams, different host threads) race on it.  Run
+ *     calls of this entry point one after another.
+ * Errors: E_NULL, E_ALIGN, E_SHAPE, E_WORKSPACE (too large for the array), E_RANGE (device index), E_CUDA. */
+int vispec_tree_verify_attn_static(const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* kv_len, const uint64_t* tree_mask, int B, int N,
+                                   int Hq, int Hkv, int D, int S_max, float scale, void* out,
+                                   float* lse, int* status_word, void* stream);
+
 /* Greedy acceptance (Sec. 3.1 at temperature 0; Table 1 upper half).  target_ids[b][i] is the
  * target model's greedy token after node i; non-root node a is matched iff
  * draft_ids[b][a] == target_ids[b][parents[b][a]]; the accepted path ends at the deepest node whose

@@ -25,7 +25,7 @@ EXPORTS = [
     "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
     "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
-    "vispec_launch_count",
+    "vispec_launch_count", "vispec_tree_verify_attn_static",
 ]
 
 
@@ -65,6 +65,7 @@ def load() -> ctypes.CDLL:
             "vispec_kv_compact": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
+            "vispec_tree_verify_attn_static": [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp],
         }
         for name, argtypes in sigs.items():
             fn = getattr(lib, name)
@@ -92,6 +93,20 @@ def _stream():
 def _check(code: int, where: str) -> None:
     if code != VISPEC_OK:
         raise VispecError(code, where)
+
+
+def tree_verify_attn_static(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                            kv_len: torch.Tensor, tree_mask: torch.Tensor, scale: float, out: torch.Tensor,
+                            lse: Optional[torch.Tensor] = None, status_word: Optional[torch.Tensor] = None) -> None:
+    """vispec_tree_verify_attn_static: the attention for callers that cannot allocate device memory
+    (no context, no workspace; scratch is a fixed array inside the library).  One C call on torch's
+    current stream; raises VispecError(VISPEC_E_WORKSPACE) when the problem exceeds the built-in scratch."""
+    B, N, Hq, D = q.shape
+    _, Hkv, S_max, _ = k_cache.shape
+    _check(load().vispec_tree_verify_attn_static(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len),
+                                                 _ptr(tree_mask), B, N, Hq, Hkv, D, S_max, ctypes.c_float(scale),
+                                                 _ptr(out), _ptr(lse), _ptr(status_word), _stream()),
+           "vispec_tree_verify_attn_static")
 
 
 class VerifyContext:
