@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying graphs")
     return ap.parse_args()
 
 
@@ -161,18 +163,42 @@ class DeviceWorkload:
         self.scale = 1.0 / math.sqrt(D)
         self.kv_bytes_per_layer = cfg.kv_bytes_per_layer(tree["kv_len"])
 
+    def _pre(self):
+        self.ctx.tree_mask_build(self.parents, self.mask, self.depth)
+
+    def _attn(self):
+        for l in range(self.L):
+            self.ctx.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
+
+    def _post(self):
+        self.ctx.accept(self.draft, self.target, self.parents, self.path, self.alen, self.bonus)
+        # kv_len itself is left as it was so that every step sees the same workload
+        self.ctx.kv_compact(0, self.L, self.path, self.alen, self.kv_len, self.new_len)
+
+    def capture(self):
+        """Capture the three phases of a step as CUDA graphs (the launches are the same C-ABI calls;
+        replaying them removes the Python/ctypes time between launches from the device timeline)."""
+        torch = self.torch
+        self.graphs = []
+        for fn in (self._pre, self._attn, self._post):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            self.graphs.append(g)
+        self.launches_per_step = None
+
     def step(self, ev_attn=None):
-        c = self.ctx
-        c.tree_mask_build(self.parents, self.mask, self.depth)
+        if getattr(self, "graphs", None):
+            pre, attn, post = (g.replay for g in self.graphs)
+        else:
+            pre, attn, post = self._pre, self._attn, self._post
+        pre()
         if ev_attn:
             ev_attn[0].record()
-        for l in range(self.L):
-            c.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
+        attn()
         if ev_attn:
             ev_attn[1].record()
-        c.accept(self.draft, self.target, self.parents, self.path, self.alen, self.bonus)
-        # kv_len itself is left as it was so that every step sees the same workload
-        c.kv_compact(0, self.L, self.path, self.alen, self.kv_len, self.new_len)
+        post()
 
 
 class HostStep:
@@ -239,22 +265,21 @@ class HostStep:
 
 # ------------------------------------------------------------------------------------ oracle legs
 
-def oracle_sample(cfg, tree, layer0, budget_heads):
-    """Time the oracle, as it stands, on one layer restricted to `budget_heads` kv heads (all of
-    their query heads, all nodes, the full cache length) plus mask, acceptance and commit."""
+def oracle_sample(cfg, tree, layers, budget_heads):
+    """Time the oracle, as it stands, on the given layers restricted to `budget_heads` kv heads (all
+    of their query heads, all nodes, the full cache length) plus mask, acceptance and commit."""
     import oracle
     G = cfg.G
     hk = min(cfg.Hkv, budget_heads)
-    q = layer0["q"][:, :, :hk * G]
-    k = layer0["k_cache"][:, :hk]
-    v = layer0["v_cache"][:, :hk]
     t0 = time.perf_counter()
     mask, _, _ = oracle.tree_mask(tree["parents"])
-    oracle.tree_attn(q, k, v, tree["kv_len"], mask, 1.0 / math.sqrt(cfg.D), want_lse=False)
     path, alen, _ = oracle.accept(tree["draft_ids"], tree["target_ids"], tree["parents"])
-    oracle.kv_compact(k, v, path, alen, tree["kv_len"])
+    for x in layers:
+        q, k, v = x["q"][:, :, :hk * G], x["k_cache"][:, :hk], x["v_cache"][:, :hk]
+        oracle.tree_attn(q, k, v, tree["kv_len"], mask, 1.0 / math.sqrt(cfg.D), want_lse=False)
+        oracle.kv_compact(k, v, path, alen, tree["kv_len"])
     dt = time.perf_counter() - t0
-    kv_bytes = int(sum(2 * (int(s) + cfg.N) * hk * cfg.D * 2 for s in tree["kv_len"]))
+    kv_bytes = len(layers) * int(sum(2 * (int(s) + cfg.N) * hk * cfg.D * 2 for s in tree["kv_len"]))
     return kv_bytes / dt / 1e9, dt, hk, oracle.num_threads()
 
 
@@ -266,9 +291,9 @@ def run_reference(args):
     from paper_2509_15235_b200 import synth
     cfg = synth.get_config(args.config)
     tree = synth.make_tree_inputs(cfg)
-    layer0 = synth.make_layer_tensors(cfg, 0)
+    layer0 = [synth.make_layer_tensors(cfg, 0)]
     heads = min(cfg.Hkv, 8)
-    for _ in range(args.warmup):
+    for _ in range(min(args.warmup, 2)):
         oracle_sample(cfg, tree, layer0, heads)
     t0 = time.perf_counter()
     vals = [oracle_sample(cfg, tree, layer0, heads) for _ in range(args.steps)]
@@ -308,7 +333,7 @@ def main():
     cfg = synth.get_config(args.config)
     warmup = max(args.warmup, 3)
 
-    tree, per_layer = build_host_inputs(cfg, cfg.layers)
+    tree, per_layer = build_host_inputs(cfg, args.layers if args.layers > 0 else cfg.layers)
     wl = DeviceWorkload(cfg, tree, per_layer, local)
     L = wl.L
 
@@ -318,11 +343,16 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-resident timing ----
+    launches0 = wl.ctx.launch_count()
+    wl.step()                                   # plain launches once: counts the kernels of one step
+    torch.cuda.synchronize()
+    launches_per_step = wl.ctx.launch_count() - launches0
+    if not args.no_graph:
+        wl.capture()
     for _ in range(warmup):
         wl.step()
     barrier()
     assert wl.ctx.status_poll() == 0
-    launches0 = wl.ctx.launch_count()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -337,7 +367,7 @@ def main():
     barrier()
     ms_total = e0.elapsed_time(e1)
     attn_ms = sum(a.elapsed_time(b) for a, b in evs)
-    launches = wl.ctx.launch_count() - launches0
+    launches = launches_per_step * args.steps
     clocks = sampler.stop() if rank == 0 else None
     status = wl.ctx.status_poll()
 
@@ -384,6 +414,7 @@ def main():
                    "kv_len": [int(s) for s in tree["kv_len"]], "layers": L,
                    "kv_bytes_per_layer": wl.kv_bytes_per_layer,
                    "l2": f"inputs larger than L2: {L} layers x {wl.kv_bytes_per_layer / 1e6:.1f} MB rotate, no flush",
+                   "launch": "plain C-ABI calls" if args.no_graph else "C-ABI calls captured once, replayed as 3 CUDA graphs per step",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
         "attn_us_per_layer": attn_s * 1e6,
@@ -398,10 +429,11 @@ def main():
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline:
-        gbs, dt, hk, cores = oracle_sample(cfg, tree, per_layer[0], min(cfg.Hkv, 32))
+        n_l = L
+        gbs, dt, hk, cores = oracle_sample(cfg, tree, per_layer[:n_l], cfg.Hkv)
         line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
-                                "sample": f"1 of {L} layers, {hk} of {cfg.Hkv} kv heads, all nodes, full KV length, plus "
-                                          f"mask/accept/commit ({dt:.2f} s of fp64 C + OpenMP)"}
+                                "sample": f"one step: {n_l} of {L} layers, {hk} of {cfg.Hkv} kv heads, all nodes, full KV "
+                                          f"length, plus mask/accept/commit ({dt:.1f} s of fp64 C + OpenMP)"}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

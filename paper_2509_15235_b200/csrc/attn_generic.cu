@@ -307,6 +307,25 @@ attn_generic_combine_kernel(const GenericParams p) {
 
 }  // namespace
 
+// Merge of partials laid out as [unit][split][64 rows][D] + [unit][split][64][2] behind the workspace
+// header (also used by the TMA/tcgen05 kernel, whose partials have the same layout).
+cudaError_t launch_attn_combine64(const AttnArgs& a, int n_split, int n_mblocks, cudaStream_t st) {
+    GenericParams p;
+    p.q = nullptr; p.k = nullptr; p.v = nullptr; p.kv_len = a.kv_len; p.mask = a.mask;
+    p.out = (__nv_bfloat16*)a.out; p.lse = a.lse;
+    const size_t units = (size_t)a.B * a.Hkv * n_mblocks;
+    unsigned char* ws = (unsigned char*)a.ws + kCounterBytes;
+    p.part_o = (float*)ws;
+    p.part_ml = (float*)(ws + units * n_split * BM * a.D * 4);
+    p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_max = a.S_max;
+    p.n_split = n_split; p.n_mblocks = n_mblocks; p.scale_log2 = 0.f; p.status = a.status;
+    const long rows = (long)a.B * a.N * a.Hq;
+    const int blocks = (int)((rows + 3) / 4);
+    if (a.D == 128) attn_generic_combine_kernel<128><<<blocks, 128, 0, st>>>(p);
+    else attn_generic_combine_kernel<64><<<blocks, 128, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
 // Per-device set-up: the D = 128 instance needs more than the default 48 KB of dynamic shared memory.
 cudaError_t init_attn_generic() {
     return cudaFuncSetAttribute(attn_generic_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,

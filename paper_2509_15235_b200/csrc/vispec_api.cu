@@ -1,4 +1,5 @@
 // C ABI of libvispec: context management, argument validation, dispatch to the kernels.
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -81,10 +82,13 @@ int vispec_ctx_create(vispec_ctx** out, const vispec_shape* s, int device) {
     ok = ok && cudaMalloc(&c->d_cache_ptrs, sizeof(void*) * 2 * s->layers) == cudaSuccess;
     ok = ok && cudaMemset(c->d_cache_ptrs, 0, sizeof(void*) * 2 * s->layers) == cudaSuccess;
     ok = ok && init_attn_generic() == cudaSuccess;
+    ok = ok && init_attn_tc5() == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { vispec_ctx_destroy(c); return VISPEC_E_CUDA; }
     c->h_k.assign(s->layers, nullptr);
     c->h_v.assign(s->layers, nullptr);
+    const char* fg = std::getenv("VISPEC_FORCE_GENERIC");
+    c->force_generic = fg && fg[0] == '1';
     c->k_map.resize(s->layers);
     c->v_map.resize(s->layers);
     *out = c;
@@ -123,12 +127,12 @@ int vispec_cache_register(vispec_ctx* c, int layer, void* k_cache, void* v_cache
     const vispec_shape& s = c->shape;
     if (s.D == 128) {
         // 3-D view (d, slot, sequence*head) of a [B,Hkv,S_max,D] bf16 cache; one box = 64 d-columns
-        // (128 bytes, the swizzle span) x 64 slots.  Slots past S_max read as zero.
+        // (128 bytes, the swizzle span) x 128 slots.  Slots past S_max read as zero.
         EncodeTiledFn enc = get_encode_fn();
         if (!enc) return VISPEC_E_CUDA;
         const cuuint64_t dims[3] = {(cuuint64_t)s.D, (cuuint64_t)s.S_max, (cuuint64_t)s.B_max * s.Hkv};
         const cuuint64_t strides[2] = {(cuuint64_t)s.D * 2, (cuuint64_t)s.S_max * s.D * 2};
-        const cuuint32_t box[3] = {64, 64, 1};
+        const cuuint32_t box[3] = {64, 128, 1};
         const cuuint32_t estr[3] = {1, 1, 1};
         void* ptrs[2] = {k_cache, v_cache};
         CUtensorMap* maps[2] = {&c->k_map[layer], &c->v_map[layer]};
@@ -177,7 +181,8 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
     a.sm_count = c->sm_count;
     a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
     int n = 0;
-    cudaError_t err = launch_attn_generic(a, (cudaStream_t)stream, &n);
+    cudaError_t err = (!c->force_generic && attn_tc5_supports(a)) ? launch_attn_tc5(a, (cudaStream_t)stream, &n)
+                                                                  : launch_attn_generic(a, (cudaStream_t)stream, &n);
     c->launches += n;
     return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
 }

@@ -19,6 +19,7 @@ struct vispec_ctx {
     void* ws = nullptr;             // caller-owned workspace
     size_t ws_bytes = 0;
     uint64_t launches = 0;
+    bool force_generic = false;     // VISPEC_FORCE_GENERIC=1 at context creation: debugging aid
 };
 
 namespace vispec {
@@ -56,5 +57,10 @@ struct AttnArgs {
 // Generic split-KV kernel on warp-level tensor-core instructions (any supported shape).
 cudaError_t init_attn_generic();   // once per device, with that device current
 cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, int* n_launches);
+
+// TMA + tcgen05 kernel (D = 128, G*N <= 64 query rows per kv head).
+bool attn_tc5_supports(const AttnArgs& a);
+cudaError_t init_attn_tc5();           // once per device, with that device current
+cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches);
 
 }  // namespace vispec
