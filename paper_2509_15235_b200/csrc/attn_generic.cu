@@ -62,6 +62,7 @@ struct GenericParams {
     __nv_bfloat16* out; float* lse;
     float* part_o; float* part_ml;      // partials: [unit][split][BM][D], [unit][split][BM][2]
     int B, N, Hq, Hkv, S_max, n_split, n_mblocks;
+    int bm;                             // rows per partial block (merge kernel only)
     float scale_log2;
     int* status;
 };
@@ -278,11 +279,11 @@ attn_generic_combine_kernel(const GenericParams p) {
     if (row >= (long)p.B * N * p.Hq) return;
     const int head = (int)(row % p.Hq), i = (int)((row / p.Hq) % N), b = (int)(row / ((long)p.Hq * N));
     const int kvh = head / G, g = head % G;
-    const int gr = i * G + g, mblk = gr / BM, lr = gr % BM;
+    const int gr = i * G + g, mblk = gr / p.bm, lr = gr % p.bm;
     const int unit = (b * p.Hkv + kvh) * p.n_mblocks + mblk;
     float m = -INFINITY;
     for (int s = 0; s < p.n_split; ++s)
-        m = fmaxf(m, p.part_ml[(((size_t)unit * p.n_split + s) * BM + lr) * 2]);
+        m = fmaxf(m, p.part_ml[(((size_t)unit * p.n_split + s) * p.bm + lr) * 2]);
     const float m_use = (m == -INFINITY) ? 0.f : m;
     constexpr int PER = D / 32;
     float acc[PER];
@@ -290,7 +291,7 @@ attn_generic_combine_kernel(const GenericParams p) {
     for (int e = 0; e < PER; ++e) acc[e] = 0.f;
     float l = 0.f;
     for (int s = 0; s < p.n_split; ++s) {
-        const size_t slot = ((size_t)unit * p.n_split + s) * BM + lr;
+        const size_t slot = ((size_t)unit * p.n_split + s) * p.bm + lr;
         const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + slot * 2);
         const float w = exp2f(ml.x - m_use);
         l += ml.y * w;
@@ -307,18 +308,18 @@ attn_generic_combine_kernel(const GenericParams p) {
 
 }  // namespace
 
-// Merge of partials laid out as [unit][split][64 rows][D] + [unit][split][64][2] behind the workspace
-// header (also used by the TMA/tcgen05 kernel, whose partials have the same layout).
-cudaError_t launch_attn_combine64(const AttnArgs& a, int n_split, int n_mblocks, cudaStream_t st) {
+// Merge of partials laid out as [unit][split][rows][D] + [unit][split][rows][2] behind the workspace header,
+// unit = (sequence * Hkv + kv head) * n_mblocks + row block.  Also used by the TMA/tcgen05 kernel.
+cudaError_t launch_attn_combine(const AttnArgs& a, int n_split, int n_mblocks, int rows_per_block, cudaStream_t st) {
     GenericParams p;
     p.q = nullptr; p.k = nullptr; p.v = nullptr; p.kv_len = a.kv_len; p.mask = a.mask;
     p.out = (__nv_bfloat16*)a.out; p.lse = a.lse;
     const size_t units = (size_t)a.B * a.Hkv * n_mblocks;
     unsigned char* ws = (unsigned char*)a.ws + kCounterBytes;
     p.part_o = (float*)ws;
-    p.part_ml = (float*)(ws + units * n_split * BM * a.D * 4);
+    p.part_ml = (float*)(ws + units * n_split * rows_per_block * a.D * 4);
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_max = a.S_max;
-    p.n_split = n_split; p.n_mblocks = n_mblocks; p.scale_log2 = 0.f; p.status = a.status;
+    p.n_split = n_split; p.n_mblocks = n_mblocks; p.bm = rows_per_block; p.scale_log2 = 0.f; p.status = a.status;
     const long rows = (long)a.B * a.N * a.Hq;
     const int blocks = (int)((rows + 3) / 4);
     if (a.D == 128) attn_generic_combine_kernel<128><<<blocks, 128, 0, st>>>(p);
@@ -354,7 +355,7 @@ cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, int* n_launc
     p.part_o = (float*)ws;
     p.part_ml = (float*)(ws + (size_t)units * n_split * BM * a.D * 4);
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_max = a.S_max;
-    p.n_split = n_split; p.n_mblocks = n_mblocks;
+    p.n_split = n_split; p.n_mblocks = n_mblocks; p.bm = BM;
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.status = a.status;
 
