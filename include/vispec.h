@@ -91,6 +91,25 @@ int vispec_workspace_bytes(const vispec_ctx* ctx, size_t* out /*host*/);
  * overlap on the GPU.  Errors: E_NULL, E_ALIGN, E_WORKSPACE (too small), E_CUDA. */
 int vispec_ctx_set_workspace(vispec_ctx* ctx, void* workspace, size_t bytes);
 
+/* Options of a context (vispec_ctx_set_option). */
+typedef enum vispec_option {
+    /* Default 1.  vispec_tree_verify_attn is enqueued so that it may start while the kernel before it on
+     * `stream` is still running (programmatic dependent launch).  Before that kernel has completed it
+     * reads only kv_len and cache tiles that lie wholly inside the committed prefix [0, S) - state that
+     * the previous decoding cycle committed; q, tree_mask, the tree's own K/V rows (slots S..S+N-1) are
+     * read, and everything is written, only after it has completed.  Set 0 if the kernel enqueued
+     * immediately before an attention call writes kv_len or committed cache slots (for instance
+     * vispec_kv_compact directly followed by attention): then nothing is read early. */
+    VISPEC_OPT_EARLY_PREFETCH = 1,
+    /* Default 0 (1 if the environment has VISPEC_FORCE_GENERIC=1 at context creation).  Route attention
+     * through the shape-generic warp-level kernel even where the TMA/tcgen05 kernel applies. */
+    VISPEC_OPT_FORCE_GENERIC = 2
+} vispec_option;
+
+/* Set an option of the context (host call, takes effect for later calls).  Errors: E_NULL,
+ * E_UNSUPPORTED (unknown option). */
+int vispec_ctx_set_option(vispec_ctx* ctx, int option, int value);
+
 /* Register layer `layer`'s cache pair [B_max,Hkv,S_max,D] bf16 (App. A: pre-allocated KV cache).
  * Builds the TMA tensor maps for these base pointers and records them for vispec_kv_compact; call
  * again if the allocator moves a cache.  Pointers must be 128-byte aligned.  Not a hot call (one

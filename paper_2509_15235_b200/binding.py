@@ -25,8 +25,10 @@ EXPORTS = [
     "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
     "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
-    "vispec_launch_count", "vispec_tree_verify_attn_static",
+    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option",
 ]
+OPT_EARLY_PREFETCH = 1
+OPT_FORCE_GENERIC = 2
 
 
 class VispecShape(ctypes.Structure):
@@ -59,6 +61,7 @@ def load() -> ctypes.CDLL:
             "vispec_workspace_bytes": [vp, ctypes.POINTER(ctypes.c_size_t)],
             "vispec_ctx_set_workspace": [vp, vp, ctypes.c_size_t],
             "vispec_cache_register": [vp, ci, vp, vp],
+            "vispec_ctx_set_option": [vp, ci, ci],
             "vispec_tree_mask_build": [vp, vp, ci, ci, vp, vp, vp],
             "vispec_tree_verify_attn": [vp, ci, vp, vp, vp, vp, vp, vp, ci, ci, cf, vp, vp, vp],
             "vispec_accept": [vp, vp, vp, vp, ci, ci, vp, vp, vp, vp],
@@ -142,6 +145,9 @@ class VerifyContext:
             self.close()
         except Exception:
             pass
+
+    def ctx_set_option(self, option: int, value: int) -> None:
+        _check(self.lib.vispec_ctx_set_option(self.handle, option, value), "vispec_ctx_set_option")
 
     # -- registration ---------------------------------------------------------------------------
     def cache_register(self, layer: int, k_cache: torch.Tensor, v_cache: torch.Tensor) -> None:

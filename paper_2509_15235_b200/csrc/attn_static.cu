@@ -76,6 +76,7 @@ extern "C" int vispec_tree_verify_attn_static(const void* q, const void* k_cache
     a.ws = s.scratch; a.ws_bytes = VISPEC_STATIC_SCRATCH_BYTES;
     a.status = status_word ? status_word : s.status;
     a.sm_count = s.sm_count;
+    a.early_prefetch = false;
     a.k_map = nullptr; a.v_map = nullptr;
     int n = 0;
     return vispec::launch_attn_generic(a, (cudaStream_t)stream, &n) == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;

@@ -1,24 +1,42 @@
 // Tree-verification attention for sm_100a (D = 128): TMA-staged K/V tiles, tcgen05 tensor-core products
 // with every accumulator AND both A operands in TMEM, fp32 online softmax (Eq. 1 restricted to prefix +
-// ancestors).
+// ancestors), work split evenly over the SMs.
 //
-// One CTA works on one (sequence, kv head, block of query rows, KV range).  Its 6 warps are specialised:
-//   warp 0     TMA producer: K ring and V ring of 128-token stages (32 KB each, 128-byte swizzle)
+// Work.  A *unit* is (sequence, kv head, block of query rows); it needs ceil((S+N)/128) *steps*, one per
+// 128 cached tokens.  All steps of all units, in the order (sequence, kv head, row block, step), form one
+// line of T steps that is cut into equal ranges, one per CTA (at most one CTA per SM; when the units are fewer
+// than the SMs the CTA count is a multiple of the unit count, so that equally long units are cut into whole
+// CTAs).  A CTA therefore runs a
+// few *segments*: the tail of one unit, whole units, the head of another.  A segment that covers its
+// whole unit writes the final bf16 output; any other writes an unnormalised partial (O, m, l) into one of
+// the CTA's two slots (first segment -> slot 2c, a later one -> slot 2c+1) and a second, small kernel merges
+// the partials of each unit.  Both kernels derive the same schedule from kv_len on the device, so the
+// host never reads lengths.
+//
+// Inside a CTA the 6 warps are specialised:
+//   warp 0     TMA producer: K ring and V ring of 128-token stages (32 KB each, 128-byte swizzle); it runs
+//              ahead across segment boundaries
 //   warp 1     tensor-core issuer (one thread): S = Q K^T and O += P V as 128x128x16 tcgen05.mma, owns TMEM
-//   warps 2-5  softmax: thread <-> TMEM lane, i.e. one thread per accumulator row, no shuffles
-// TMEM map (512 columns x 128 lanes): S[0] 0..127, S[1] 128..255, O 256..383, Q 384..447.
-// Q (bf16, packed two per column) is written to TMEM once by the softmax threads and is the A operand of
-// every S product; P (bf16) overwrites the first 64 columns of the S buffer it came from and is the A
-// operand of the PV product, so neither Q nor P ever touches shared memory: all of it goes to the rings.
+//   warps 2-5  softmax: thread <-> TMEM lane, i.e. one thread per accumulator row, no shuffles; they also
+//              load Q at the start of every segment and run the segment epilogue
+// TMEM map (512 columns x 128 lanes): S[0] 0..127, S[1] 128..255, O 256..383, Q 384..447, P 448..511.
+// Q and P (bf16, packed two per column) are the A operands of the S and PV products, so neither ever
+// touches shared memory.  S is double-buffered and released as soon as the softmax threads have read it,
+// so the S product of step u+1 runs while step u is in the softmax.
 //
 // Two row layouts share the code:
 //   FULL  (G*N > 64):  lane r holds query row r of the block; a thread handles all 128 tokens of a step.
 //   PAIR  (G*N <= 64): the <= 64 query rows are duplicated, lanes 0-63 take tokens 0-63 of each step and
 //                      lanes 64-127 tokens 64-127 (P is block-diagonal); the two halves keep independent
-//                      softmax states and are merged once in the epilogue.  All 128 threads stay busy and
-//                      the tensor core runs full-height instructions, which cost less than two 64-row ones.
+//                      softmax states and are merged once per segment through shared memory.
 // The running maximum is only moved when a tile exceeds it by more than 2^8 (O and l share the reference, so
 // the result is exact either way); O is therefore re-scaled in TMEM rarely.
+//
+// Programmatic dependent launch: both kernels are launched with programmatic stream serialisation.  The
+// attention kernel reads kv_len and (when early prefetch is on) streams K/V tiles that lie wholly inside the
+// committed prefix before it waits for the preceding kernel; q, tree_mask, the tree's own K/V rows and every
+// write come after that wait.
+//
 // Every wait on an mbarrier is bounded; on a timeout the CTA records VISPEC_E_TIMEOUT, drains its own
 // copies, frees its TMEM and returns.
 #include <cuda_bf16.h>
@@ -27,30 +45,42 @@
 
 namespace vispec {
 
-cudaError_t launch_attn_combine(const AttnArgs& a, int n_split, int n_mblocks, int rows_per_block, cudaStream_t st);
-
 namespace {
 
 constexpr int D = 128;
 constexpr int STEP = 128;                      // tokens per pipeline step = rows of one K or V stage
 constexpr int HALF_BYTES = STEP * 128;         // one d-half (64 columns) of a stage: 128 rows x 128 B
 constexpr int STAGE_BYTES = 2 * HALF_BYTES;    // 32 KB
-constexpr int NSK = 3, NSV = 4;
+constexpr int NSK = 3, NSV = 3;
 constexpr int kThreads = 192;
+constexpr int kMaxB = 64;                      // sequences per call this kernel takes
 constexpr int SMEM_K = 0;
 constexpr int SMEM_V = SMEM_K + NSK * STAGE_BYTES;
-constexpr int SMEM_BAR = SMEM_V + NSV * STAGE_BYTES;
-constexpr int SMEM_TOTAL = SMEM_BAR + 256;
-constexpr int SMEM_ALLOC = SMEM_TOTAL + 1024;                  // slack to align the base to 1024 B
+constexpr int SMEM_X = SMEM_V + NSV * STAGE_BYTES;             // PAIR exchange: [32 col4][64 rows] float4 + 64 float2
+constexpr int X_BYTES = 32 * 64 * 16 + 64 * 8;
+constexpr int SMEM_BAR = SMEM_X + X_BYTES;
+constexpr int BAR_BYTES = 256;
+constexpr int SMEM_SCHED = SMEM_BAR + BAR_BYTES;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t COL_S = 0, COL_O = 256, COL_Q = 384;
+constexpr uint32_t COL_S = 0, COL_O = 256, COL_Q = 384, COL_P = 448;
 constexpr float kRescaleGap = 8.0f;                            // log2 units
 constexpr long long kWaitCycles = 1500000000LL;                // ~0.8 s at 1.9 GHz
 
 enum { B_KFULL = 0, B_KEMPTY = B_KFULL + NSK, B_VFULL = B_KEMPTY + NSK, B_VEMPTY = B_VFULL + NSV,
-       B_SFULL = B_VEMPTY + NSV, B_PFULL = B_SFULL + 2, B_PVDONE = B_PFULL + 2,
-       B_XSTAT = B_PVDONE + 2, B_XWGT = B_XSTAT + 1, B_XCH = B_XWGT + 1, B_COUNT = B_XCH + 4 };
-static_assert(B_COUNT * 8 + 16 <= 256, "barrier block too small");
+       B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 1,
+       B_QFULL = B_PVDONE + 1, B_XCH = B_QFULL + 1, B_XFREE = B_XCH + 1, B_COUNT = B_XFREE + 1 };
+static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block too small");
+
+// The schedule every CTA (and the merge kernel) derives from kv_len.
+struct Sched {
+    int base[kMaxB + 1];   // first global step of sequence b; base[B] = T
+    int steps[kMaxB];      // steps of one unit of sequence b (0: sequence rejected or empty)
+    int len[kMaxB];        // committed length S of sequence b
+    int units;             // units with at least one step
+};
+constexpr int SMEM_TOTAL = SMEM_SCHED + (int)sizeof(Sched);
+constexpr int SMEM_ALLOC = SMEM_TOTAL + 1024;                  // slack to align the base to 1024 B
+static_assert(SMEM_ALLOC <= 232448, "over the 227 KB a CTA may have");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -100,6 +130,9 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// Programmatic dependent launch: let the next kernel in the stream be scheduled / wait for the previous one.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // One tcgen05.mma (cta_group::1, kind::f16) with the A operand in TMEM and B described in shared memory.
 // The 64-bit descriptor is passed as 32-bit halves: the high half is constant, the low half carries the address.
 __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
@@ -151,18 +184,41 @@ __host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) {
 __host__ __device__ constexpr uint32_t instr_desc(int b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
+// 128-bit shifts on (lo, hi) pairs; any shift count >= 0.
+__device__ __forceinline__ void shr128(uint64_t lo, uint64_t hi, int s, uint64_t& rlo, uint64_t& rhi) {
+    if (s >= 128) { rlo = 0; rhi = 0; }
+    else if (s >= 64) { rlo = hi >> (s - 64); rhi = 0; }
+    else if (s == 0) { rlo = lo; rhi = hi; }
+    else { rlo = (lo >> s) | (hi << (64 - s)); rhi = hi >> s; }
+}
+__device__ __forceinline__ void shl128_fill(uint64_t lo, uint64_t hi, int s, uint64_t& rlo, uint64_t& rhi) {
+    // shift left by s in (0, 128) and set the s vacated low bits
+    if (s >= 64) { rlo = ~0ull; rhi = (lo << (s - 64)) | (s == 64 ? 0ull : ((1ull << (s - 64)) - 1)); }
+    else { rlo = (lo << s) | ((1ull << s) - 1); rhi = (hi << s) | (lo >> (64 - s)); }
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
 #ifdef VISPEC_TC5_TRACE
-// Debug build only: CTA (0,0) logs clock64() stamps per role and step: g_trace[role][step][slot].
+// Debug build only: CTA 0 logs clock64() stamps per role and step: g_trace[role][step][slot].
 __device__ long long g_trace[3][64][8];
 __device__ long long g_trace_misc[16];
-#define TRACE(role, step, slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) < 64) g_trace[role][step][slot] = clock64(); } while (0)
-#define TRACE_MISC(slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 64) g_trace_misc[slot] = clock64(); } while (0)
+__device__ int g_trace_cta = 0;
+#define TRACE(role, step, slot) do { if (blockIdx.x == g_trace_cta && (step) < 64) g_trace[role][step][slot] = clock64(); } while (0)
+#define TRACE_MISC(slot) do { if (blockIdx.x == g_trace_cta && threadIdx.x == 64) g_trace_misc[slot] = clock64(); } while (0)
+// Per-launch timeline in globaltimer nanoseconds: [launch][0/1] attention first start / last end, [2/3] merge.
+__device__ unsigned long long g_timeline[4096][4];
+__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+__device__ unsigned long long g_cta_times[256][4];
+#define CTA_T(k) do { if (threadIdx.x == 0 && blockIdx.x < 256) g_cta_times[blockIdx.x][k] = gtimer(); } while (0)
+#define TL_START(idx, k) do { if (threadIdx.x == 0 && (idx) < 4096) atomicMin(&g_timeline[idx][k], gtimer()); } while (0)
+#define TL_END(idx, k) do { if (threadIdx.x == 0 && (idx) < 4096) atomicMax(&g_timeline[idx][k], gtimer()); } while (0)
 #else
+#define CTA_T(k) do {} while (0)
+#define TL_START(idx, k) do {} while (0)
+#define TL_END(idx, k) do {} while (0)
 #define TRACE(role, step, slot) do {} while (0)
 #define TRACE_MISC(slot) do {} while (0)
 #endif
@@ -170,10 +226,94 @@ __device__ long long g_trace_misc[16];
 struct Tc5Params {
     const __nv_bfloat16* q; const int32_t* kv_len; const uint64_t* mask;
     __nv_bfloat16* out; float* lse;
-    float* part_o; float* part_ml;        // [unit][split][ROWS][D], [unit][split][ROWS][2]
-    int B, N, Hq, Hkv, S_max, n_split, n_mblocks;
+    float4* part_o;            // [slot][32 col4][ROWS]: column-of-4 major, so that a warp's 32 rows are contiguous
+    float2* part_ml;           // [slot][ROWS]: (m in log2 units or -inf, l)
+    int B, N, Hq, Hkv, S_max, n_mblocks;
+    int grid_attn;             // CTAs of the attention kernel (the merge kernel needs it for the schedule)
+    int min_steps;             // a CTA is given at least this many steps (fewer CTAs work on small problems)
+    int early;                 // stream committed-prefix tiles before waiting for the preceding kernel
     float scale_log2;
     int* status;
+    int trace_idx;             // launch index (trace builds only)
+};
+
+// ---- schedule ---------------------------------------------------------------------------------------
+// Built by one full warp.  Reads kv_len only.
+__device__ void sched_build(Sched& s, const Tc5Params& p, int lane) {
+    const int upb = p.Hkv * p.n_mblocks;        // units per sequence
+    int carry = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+        const int b = b0 + lane;
+        int st = 0, S = 0;
+        if (b < p.B) {
+            S = p.kv_len[b];
+            const bool ok = (S >= 0 && S + p.N <= p.S_max);
+            st = ok ? (S + p.N + STEP - 1) / STEP : 0;
+            s.steps[b] = st;
+            s.len[b] = S;
+        }
+        int x = st * upb;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (b < p.B) s.base[b] = carry + x - st * upb;
+        carry += __shfl_sync(0xffffffffu, x, 31);
+    }
+    if (lane == 0) s.base[p.B] = carry;
+    __syncwarp();
+    int live = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+        const int b = b0 + lane;
+        live += __popc(__ballot_sync(0xffffffffu, b < p.B && s.steps[b] > 0));
+    }
+    if (lane == 0) s.units = live * upb;
+}
+// Number of CTAs that get work: every CTA at least min_steps steps; a multiple of the unit count when
+// the units are fewer than the CTAs (equally long units then never share a CTA).
+__device__ __forceinline__ int sched_ctas(int T, int units, int grid, int min_steps) {
+    int g = T / min_steps;
+    g = g < 1 ? 1 : g;
+    g = g < grid ? g : grid;
+    if (units <= g) g = (g / units) * units;
+    return g;
+}
+// (T * grid < 2^31 is checked on the host, so 32-bit arithmetic suffices)
+__device__ __forceinline__ int cta_lo(int c, int T, int geff) { return (int)(((unsigned)c * (unsigned)T) / (unsigned)geff); }
+// The CTA whose range holds global step g.
+__device__ __forceinline__ int cta_of(int g, int T, int geff) {
+    int c = (int)((((unsigned)g + 1u) * (unsigned)geff - 1u) / (unsigned)T);
+    c = c > geff - 1 ? geff - 1 : c;
+    while (cta_lo(c, T, geff) > g) --c;
+    while (c + 1 < geff && cta_lo(c + 1, T, geff) <= g) ++c;
+    return c;
+}
+
+struct Seg {
+    int b, kvh, mblock, st0, n, steps, S, slot;    // slot < 0: the segment is a whole unit
+};
+struct SegIter {
+    const Sched* s;
+    int B, n_mblocks, g, lo, hi, cta;
+    __device__ __forceinline__ bool next(Seg& o) {
+        if (g >= hi) return false;
+        int l = 0, r = B;                               // first b with base[b] > g, minus one
+        while (l < r) { const int m = (l + r) >> 1; if (s->base[m] <= g) l = m + 1; else r = m; }
+        o.b = l - 1;
+        o.steps = s->steps[o.b];
+        o.S = s->len[o.b];
+        const int rel = g - s->base[o.b];
+        const int uib = rel / o.steps;
+        o.st0 = rel - uib * o.steps;
+        o.n = min(hi - g, o.steps - o.st0);
+        o.kvh = uib / n_mblocks;
+        o.mblock = uib - o.kvh * n_mblocks;
+        const bool whole = (o.st0 == 0 && o.n == o.steps);
+        o.slot = whole ? -1 : (g == lo ? 2 * cta : 2 * cta + 1);
+        g += o.n;
+        return true;
+    }
 };
 
 template <bool PAIR>
@@ -183,71 +323,182 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     constexpr int NCOL = PAIR ? 64 : 128;      // tokens of a step one thread handles
     extern __shared__ unsigned char smem_raw[];
     TRACE_MISC(0);
+    TL_START(p.trace_idx, 0);
+    CTA_T(0);
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* sm = smem_raw + (base - raw);
     const uint32_t bars = base + SMEM_BAR;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + SMEM_BAR + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SMEM_BAR + B_COUNT * 8 + 8);
+    Sched& sched = *reinterpret_cast<Sched*>(sm + SMEM_SCHED);
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int split = blockIdx.x, unit = blockIdx.y;
-    const int mblock = unit % p.n_mblocks, bh = unit / p.n_mblocks;       // bh = sequence * Hkv + kv head
-    const int b = bh / p.Hkv, kvh = bh % p.Hkv;
+    const int cta = blockIdx.x;
     const int G = p.Hq / p.Hkv, N = p.N, W = (N + 63) >> 6;
     const int rows_total = G * N;
-
-    const int S = p.kv_len[b];
-    const bool seq_ok = (S >= 0 && S + N <= p.S_max);
-    if (!seq_ok && tid == 0 && split == 0 && mblock == 0) atomicCAS(p.status, 0, (int)VISPEC_E_RANGE);
-    const int total = seq_ok ? S + N : 0;
-    const int steps_total = (total + STEP - 1) / STEP;
-    const int sps = (steps_total + p.n_split - 1) / p.n_split;
-    const int step_begin = min(split * sps, steps_total);
-    const int nsteps = min(step_begin + sps, steps_total) - step_begin;
-    const int tok_begin = step_begin * STEP;
-
-    // row handled by this thread if it is a softmax thread (warps 2..5 cover the four TMEM lane quarters)
-    const int sp = warp & 3;
-    const int tl = sp * 32 + lane;                       // TMEM lane
-    const int half = PAIR ? (tl >> 6) : 0;               // PAIR: which 64 tokens of each step
-    const int lrow = PAIR ? (tl & 63) : tl;              // row within the block
-    const int row = mblock * 128 + lrow;                 // query row within the kv head's G*N rows
-    const bool row_ok = row < rows_total;
-    const int node = row_ok ? row / G : 0, head = kvh * G + (row_ok ? row % G : 0);
 
     if (tid == 0) {
         for (int i = 0; i < NSK; ++i) { mbar_init(bar(B_KFULL + i), 1); mbar_init(bar(B_KEMPTY + i), 1); }
         for (int i = 0; i < NSV; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(B_SFULL + i), 1); mbar_init(bar(B_PFULL + i), 128); mbar_init(bar(B_PVDONE + i), 1);
+            mbar_init(bar(B_SFULL + i), 1); mbar_init(bar(B_SFREE + i), 128);
         }
-        for (int i = B_XSTAT; i < B_COUNT; ++i) mbar_init(bar(i), 64);
+        mbar_init(bar(B_PFULL), 128); mbar_init(bar(B_PVDONE), 1); mbar_init(bar(B_QFULL), 128);
+        mbar_init(bar(B_XCH), 64); mbar_init(bar(B_XFREE), 64);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (nsteps > 0 && warp == 1) {
+    if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    if (warp == 2) sched_build(sched, p, lane);
+    pdl_launch_dependents();
+    if (!p.early) pdl_wait();
     TRACE_MISC(1);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     TRACE_MISC(2);
 
-    float m_ref = -INFINITY, l_run = 0.f;
-    bool has_o = false;
+    const int T = sched.base[p.B];
+    const int geff = T > 0 ? sched_ctas(T, sched.units, (int)gridDim.x, p.min_steps) : 0;
+    const bool active = cta < geff;
+    const int lo = active ? cta_lo(cta, T, geff) : 0, hi = active ? cta_lo(cta + 1, T, geff) : 0;
+    const uint32_t tmem = *tmem_slot;
+    auto make_iter = [&]() { SegIter it; it.s = &sched; it.B = p.B; it.n_mblocks = p.n_mblocks; it.g = lo; it.lo = lo; it.hi = hi; it.cta = cta; return it; };
 
-    if (nsteps > 0) {
-        const uint32_t tmem = *tmem_slot;
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0 && active) {
+            bool waited = !p.early;
+            int it = 0, nk = 0, nv = 0;          // steps started; K / V stages issued
+            bool ok = true;
+            SegIter si = make_iter();
+            Seg sg;
+            while (ok && si.next(sg)) {
+                const int bh = sg.b * p.Hkv + sg.kvh;
+                for (int t = 0; t < sg.n; ++t, ++it) {
+                    const int tok = (sg.st0 + t) * STEP;
+                    if (!waited && tok + STEP > sg.S) { pdl_wait(); waited = true; }   // the tree's rows come from the preceding kernel
+                    const int sk = it % NSK, sv = it % NSV;
+                    TRACE(0, it, 0);
+                    if (!mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    TRACE(0, it, 1);
+                    mbar_expect_tx(bar(B_KFULL + sk), STAGE_BYTES);
+                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES, &k_map, bar(B_KFULL + sk), 0, tok, bh);
+                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES, &k_map, bar(B_KFULL + sk), 64, tok, bh);
+                    ++nk;
+                    if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    TRACE(0, it, 2);
+                    mbar_expect_tx(bar(B_VFULL + sv), STAGE_BYTES);
+                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES, &v_map, bar(B_VFULL + sv), 0, tok, bh);
+                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES, &v_map, bar(B_VFULL + sv), 64, tok, bh);
+                    ++nv;
+                }
+            }
+            if (*abort_flag) {
+                // drain: wait (bounded, fresh timer) until every copy this thread issued has landed
+                volatile int never = 0;
+                for (int u = max(0, nk - NSK); u < nk; ++u) mbar_wait(bar(B_KFULL + u % NSK), (u / NSK) & 1, &never);
+                for (int u = max(0, nv - NSV); u < nv; ++u) mbar_wait(bar(B_VFULL + u % NSV), (u / NSV) & 1, &never);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ================= tensor-core issuer =================
+        if (lane == 0 && active) {
+            constexpr uint32_t IDESC_S = instr_desc(0);            // B = K stage, K-major
+            constexpr uint32_t IDESC_O = instr_desc(1);            // B = V stage, MN-major
+            constexpr uint32_t DESC_HI = desc_hi(1024);            // 8 rows x 128 B between row groups, everywhere
+            auto issue_pv = [&](int u, uint32_t acc) -> bool {
+                const int sv = u % NSV;
+                TRACE(1, u, 3);
+                if (!mbar_wait(bar(B_PFULL), u & 1, abort_flag)) return false;
+                TRACE(1, u, 4);
+                if (!mbar_wait(bar(B_VFULL + sv), (u / NSV) & 1, abort_flag)) return false;
+                TRACE(1, u, 5);
+                tc_fence_after();
+                const uint32_t vb = desc_lo(base + SMEM_V + sv * STAGE_BYTES, HALF_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < STEP / 16; ++ks)      // 16 tokens per instruction: 8 P columns, 16 V rows (2 KB)
+                    tc_mma_ts(tmem + COL_O, tmem + COL_P + ks * 8, vb + ks * 128, DESC_HI, IDESC_O,
+                              (acc || ks > 0) ? 1u : 0u);
+                tc_commit(bar(B_VEMPTY + sv));
+                tc_commit(bar(B_PVDONE));
+                TRACE(1, u, 6);
+                return true;
+            };
+            bool ok = true, have_prev = false;
+            uint32_t acc_prev = 0;
+            int it = 0, seg = 0;
+            SegIter si = make_iter();
+            Seg sg;
+            while (ok && si.next(sg)) {
+                // Q of this segment is loaded only after the previous segment's epilogue, which waits for that
+                // segment's last PV product: issue it before waiting for Q
+                if (have_prev) { ok = issue_pv(it - 1, acc_prev); have_prev = false; if (!ok) break; }
+                if (!mbar_wait(bar(B_QFULL), seg & 1, abort_flag)) { ok = false; break; }
+                for (int t = 0; t < sg.n && ok; ++t, ++it) {
+                    const int bs = it & 1, sk = it % NSK;
+                    TRACE(1, it, 0);
+                    if (!mbar_wait(bar(B_KFULL + sk), (it / NSK) & 1, abort_flag)) { ok = false; break; }
+                    TRACE(1, it, 1);
+                    // S[bs] is free once the softmax threads have read the scores of step it-2 out of it
+                    if (it >= 2 && !mbar_wait(bar(B_SFREE + bs), ((it >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t kb = desc_lo(base + SMEM_K + sk * STAGE_BYTES, 16);
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks)         // 16 d-columns per instruction: 8 Q columns, 32 B of each K row
+                        tc_mma_ts(tmem + COL_S + bs * 128, tmem + COL_Q + ks * 8,
+                                  kb + (((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4), DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+                    tc_commit(bar(B_KEMPTY + sk));
+                    tc_commit(bar(B_SFULL + bs));
+                    TRACE(1, it, 2);
+                    if (have_prev) ok = issue_pv(it - 1, acc_prev);
+                    have_prev = true;
+                    acc_prev = t > 0 ? 1u : 0u;                 // the first product of a segment starts a fresh O
+                }
+                ++seg;
+            }
+            if (ok && have_prev) issue_pv(it - 1, acc_prev);
+        }
+        __syncwarp();
+    } else {
+        // ================= softmax: one thread per accumulator row =================
+        const int sp = warp & 3;
+        const int tl = sp * 32 + lane;                       // TMEM lane
+        const int half = PAIR ? (tl >> 6) : 0;               // PAIR: which 64 tokens of each step
+        const int lrow = PAIR ? (tl & 63) : tl;              // row within the block
         const uint32_t lane_addr = tmem + ((uint32_t)(32 * sp) << 16);
-        // ---- Q -> TMEM: each softmax thread packs its row (bf16 pairs) into columns COL_Q..COL_Q+63 ----
-        if (warp >= 2) {
+        const int st = tid - 64;                              // 0..127
+        pdl_wait();                                           // q, tree_mask and every output come after the preceding kernel
+
+        // rejected sequences (kv_len < 0 or kv_len + N > S_max): zero output, -inf lse, status word
+        {
+            bool any_bad = false;
+            for (int b = 0; b < p.B; ++b) {
+                const int S = sched.len[b];
+                if (S >= 0 && S + N <= p.S_max) continue;
+                any_bad = true;
+                const int vecs = N * p.Hq * (D / 8);
+                uint4* o = reinterpret_cast<uint4*>(p.out + (size_t)b * N * p.Hq * D);
+                for (int i = cta * 128 + st; i < vecs; i += (int)gridDim.x * 128) o[i] = make_uint4(0, 0, 0, 0);
+                if (p.lse)
+                    for (int i = cta * 128 + st; i < N * p.Hq; i += (int)gridDim.x * 128) p.lse[(size_t)b * p.Hq * N + i] = -INFINITY;
+            }
+            if (any_bad && cta == 0 && st == 0) atomicCAS(p.status, 0, (int)VISPEC_E_RANGE);
+        }
+
+        // Q of a segment -> TMEM buffer `buf`: each thread packs its row (bf16 pairs) into 64 columns
+        auto load_q = [&](const Seg& sg) {
+            const int row = sg.mblock * 128 + lrow;
             uint32_t qreg[64];
-            if (row_ok) {
-                const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)b * N + node) * p.Hq + head) * D);
+            if (row < rows_total) {
+                const int node = row / G, head = sg.kvh * G + row % G;
+                const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)sg.b * N + node) * p.Hq + head) * D);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     const uint4 v4 = src[c];
@@ -260,327 +511,328 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             tmem_st32(lane_addr + COL_Q, qreg);
             tmem_st32(lane_addr + COL_Q + 32, qreg + 32);
             tmem_wait_st();
-        }
-        TRACE_MISC(3);
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        TRACE_MISC(4);
+            tc_fence_before();
+            mbar_arrive(bar(B_QFULL));
+        };
 
-        if (warp == 0) {
-            // ================= TMA producer =================
-            if (lane == 0) {
-                int issued = 0;
-                for (int t = 0; t < nsteps; ++t) {
-                    const int tok = tok_begin + t * STEP;
-                    const int sk = t % NSK, sv = t % NSV;
-                    TRACE(0, t, 0);
-                    if (!mbar_wait(bar(B_KEMPTY + sk), ((t / NSK) & 1) ^ 1, abort_flag)) break;
-                    TRACE(0, t, 1);
-                    mbar_expect_tx(bar(B_KFULL + sk), STAGE_BYTES);
-                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES, &k_map, bar(B_KFULL + sk), 0, tok, bh);
-                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES, &k_map, bar(B_KFULL + sk), 64, tok, bh);
-                    if (!mbar_wait(bar(B_VEMPTY + sv), ((t / NSV) & 1) ^ 1, abort_flag)) { issued = -(t + 1); break; }
-                    TRACE(0, t, 2);
-                    mbar_expect_tx(bar(B_VFULL + sv), STAGE_BYTES);
-                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES, &v_map, bar(B_VFULL + sv), 0, tok, bh);
-                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES, &v_map, bar(B_VFULL + sv), 64, tok, bh);
-                    issued = t + 1;
-                }
-                if (*abort_flag) {
-                    // drain: wait (bounded, fresh timer) until every copy this thread issued has landed
-                    volatile int never = 0;
-                    const int nk = issued < 0 ? -issued : issued, nv = issued < 0 ? -issued - 1 : issued;
-                    for (int u = max(0, nk - NSK); u < nk; ++u) mbar_wait(bar(B_KFULL + u % NSK), (u / NSK) & 1, &never);
-                    for (int u = max(0, nv - NSV); u < nv; ++u) mbar_wait(bar(B_VFULL + u % NSV), (u / NSV) & 1, &never);
-                }
-            }
-            __syncwarp();
-        } else if (warp == 1) {
-            // ================= tensor-core issuer =================
-            if (lane == 0) {
-                constexpr uint32_t IDESC_S = instr_desc(0);            // B = K stage, K-major
-                constexpr uint32_t IDESC_O = instr_desc(1);            // B = V stage, MN-major
-                constexpr uint32_t DESC_HI = desc_hi(1024);            // 8 rows x 128 B between row groups, everywhere
-                auto issue_pv = [&](int u) -> bool {
-                    const int bu = u & 1, sv = u % NSV;
-                    TRACE(1, u, 3);
-                    if (!mbar_wait(bar(B_PFULL + bu), (u >> 1) & 1, abort_flag)) return false;
-                    TRACE(1, u, 4);
-                    if (!mbar_wait(bar(B_VFULL + sv), (u / NSV) & 1, abort_flag)) return false;
-                    TRACE(1, u, 5);
-                    tc_fence_after();
-                    const uint32_t vb = desc_lo(base + SMEM_V + sv * STAGE_BYTES, HALF_BYTES);
-#pragma unroll
-                    for (int ks = 0; ks < STEP / 16; ++ks)      // 16 tokens per instruction: 8 P columns, 16 V rows (2 KB)
-                        tc_mma_ts(tmem + COL_O, tmem + COL_S + bu * 128 + ks * 8, vb + ks * 128, DESC_HI, IDESC_O,
-                                  (u > 0 || ks > 0) ? 1u : 0u);
-                    tc_commit(bar(B_VEMPTY + sv));
-                    tc_commit(bar(B_PVDONE + bu));
-                    TRACE(1, u, 6);
-                    return true;
-                };
-                bool ok = true;
-                for (int t = 0; t < nsteps && ok; ++t) {
-                    const int bs = t & 1, sk = t % NSK;
-                    TRACE(1, t, 0);
-                    if (!mbar_wait(bar(B_KFULL + sk), (t / NSK) & 1, abort_flag)) { ok = false; break; }
-                    TRACE(1, t, 1);
-                    // S[bs] (and the P that aliases it) is free once the PV product of step t-2 has completed
-                    if (t >= 2 && !mbar_wait(bar(B_PVDONE + bs), ((t >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t kb = desc_lo(base + SMEM_K + sk * STAGE_BYTES, 16);
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)         // 16 d-columns per instruction: 8 Q columns, 32 B of each K row
-                        tc_mma_ts(tmem + COL_S + bs * 128, tmem + COL_Q + ks * 8,
-                                  kb + (((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4), DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
-                    tc_commit(bar(B_KEMPTY + sk));
-                    tc_commit(bar(B_SFULL + bs));
-                    TRACE(1, t, 2);
-                    if (t >= 1) ok = issue_pv(t - 1);
-                }
-                if (ok) issue_pv(nsteps - 1);
-            }
-            __syncwarp();
-        } else {
-            // ================= softmax: one thread per accumulator row =================
-            uint64_t mk0 = 0, mk1 = 0;
-            if (row_ok) {
-                const uint64_t* mrow = p.mask + ((size_t)b * N + node) * W;
-                mk0 = mrow[0];
-                if (W > 1) mk1 = mrow[1];
-            }
+        if (active) {
+            SegIter si = make_iter();
+            Seg sg;
+            int it = 0, seg = 0;
             bool ok = true;
-            for (int t = 0; t < nsteps; ++t) {
-                const int bs = t & 1;
-                if (tid == 64) TRACE(2, t, 0);
-                if (!mbar_wait_warp(bar(B_SFULL + bs), (t >> 1) & 1, abort_flag)) { ok = false; break; }
-                if (tid == 64) TRACE(2, t, 1);
-                tc_fence_after();
-                uint32_t sraw[NCOL];
-#pragma unroll
-                for (int ch = 0; ch < NCOL / 32; ++ch) tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + ch * 32, sraw + ch * 32);
-                tmem_wait_ld();
-                if (tid == 64) TRACE(2, t, 2);
+            float4* xch = reinterpret_cast<float4*>(sm + SMEM_X);
+            float2* xst = reinterpret_cast<float2*>(sm + SMEM_X + 32 * 64 * 16);
+            while (ok && si.next(sg)) {
+                // every S product of the previous segment has been consumed by now, so Q may be replaced
+                load_q(sg);
+                TRACE_MISC(3);
 
-                const int j0 = tok_begin + t * STEP + half * 64;        // first token this thread looks at
-                const bool valid = j0 < total;
-                float tmax = -INFINITY;
-                if (valid) {
+                const int row = sg.mblock * 128 + lrow;          // query row within the kv head's G*N rows
+                const bool row_ok = row < rows_total;
+                const int node = row_ok ? row / G : 0, head = sg.kvh * G + (row_ok ? row % G : 0);
+                const int S = sg.S, total = S + N;
+                uint64_t mk0 = 0, mk1 = 0;
+                if (row_ok) {
+                    const uint64_t* mrow = p.mask + ((size_t)sg.b * N + node) * W;
+                    mk0 = mrow[0];
+                    if (W > 1) mk1 = mrow[1];
+                    // bits at or beyond N are not tree nodes
+                    if (N < 64) mk0 &= (1ull << N) - 1;
+                    if (N < 128) mk1 &= N > 64 ? (1ull << (N - 64)) - 1 : 0ull;
+                }
+                float m_ref = -INFINITY, l_run = 0.f;
+                bool has_o = false;
+
+                for (int t = 0; t < sg.n; ++t, ++it) {
+                    const int bs = it & 1;
+                    const int tok0 = (sg.st0 + t) * STEP;
+                    if (tid == 64) TRACE(2, it, 0);
+                    if (!mbar_wait_warp(bar(B_SFULL + bs), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (tid == 64) TRACE(2, it, 1);
+                    tc_fence_after();
+                    uint32_t sraw[NCOL];
 #pragma unroll
-                    for (int c = 0; c < NCOL; ++c) sraw[c] = __float_as_uint(__uint_as_float(sraw[c]) * p.scale_log2);
-                    if (j0 + NCOL > S) {
-                        // reaches past the committed prefix: ancestor bits for tree rows, nothing beyond them
-                        const int t0 = j0 - S;                           // tree index of column 0 (may be negative)
+                    for (int ch = 0; ch < NCOL / 32; ++ch) tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + ch * 32, sraw + ch * 32);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    mbar_arrive(bar(B_SFREE + bs));             // the S product of step it+2 may overwrite the buffer
+                    if (tid == 64) TRACE(2, it, 2);
+
+                    const int j0 = tok0 + half * 64;                        // first token this thread looks at
+                    const bool valid = j0 < total;
+                    float tmax = -INFINITY;
+                    if (valid) {
+                        if (j0 + NCOL > S) {
+                            // reaches past the committed prefix: ancestor bits for tree rows, nothing beyond them
+                            // bit c of (a0, a1): column c may be attended to (prefix column, or visible tree node)
+                            const int t0 = j0 - S;                           // tree index of column 0 (may be negative)
+                            uint64_t a0, a1;
+                            if (t0 >= 0) shr128(mk0, mk1, t0, a0, a1); else shl128_fill(mk0, mk1, -t0, a0, a1);
 #pragma unroll
-                        for (int c = 0; c < NCOL; ++c) {
-                            const int tt = t0 + c;
-                            bool allow = true;
-                            if (tt >= 0) allow = (tt < N) && ((tt < 64 ? (mk0 >> tt) : (mk1 >> (tt - 64))) & 1ull);
-                            if (!allow) sraw[c] = 0xff800000u;          // -inf
+                            for (int c = 0; c < NCOL; ++c)
+                                if (!(((c < 64 ? a0 : a1) >> (c & 63)) & 1ull)) sraw[c] = 0xff800000u;   // -inf
+                        }
+                        float mx[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sraw[c]);
+#pragma unroll
+                        for (int c = 8; c < NCOL; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sraw[c]));
+                        // the scale is positive, so it commutes with the maximum
+                        tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
+                    }
+                    // move the reference maximum only when the tile exceeds it by more than the gap
+                    float alpha = 1.f;
+                    bool rescale = false;
+                    if (valid && tmax > m_ref + kRescaleGap) {          // also true on the first finite tile (m_ref = -inf)
+                        alpha = exp2f(m_ref - tmax);                     // 0 when m_ref = -inf
+                        m_ref = tmax;
+                        l_run *= alpha;
+                        rescale = has_o;
+                    }
+                    // the PV product of step it-1 must be complete before P is replaced (and before O is touched)
+                    if (it >= 1) {
+                        if (!mbar_wait_warp(bar(B_PVDONE), (it - 1) & 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                    }
+                    if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t o[32];
+                            tmem_ld32(lane_addr + COL_O + ch * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            tmem_st32(lane_addr + COL_O + ch * 32, o);
                         }
                     }
-                    float mx[8];
+                    if (tid == 64) TRACE(2, it, 3);
+                    // P = exp2(scale * s - m_ref) as bf16 pairs into the P columns (column c holds tokens 2c, 2c+1)
+                    uint32_t pd[NCOL / 2];
+                    if (valid) {
+                        const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                        float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sraw[c]);
+                        for (int c = 0; c < NCOL / 2; ++c) {
+                            const float e0 = exp2f(fmaf(__uint_as_float(sraw[2 * c]), p.scale_log2, -m_use));
+                            const float e1 = exp2f(fmaf(__uint_as_float(sraw[2 * c + 1]), p.scale_log2, -m_use));
+                            sum0 += e0; sum1 += e1;
+                            pd[c] = pack_bf16(e0, e1);
+                        }
+                        l_run += sum0 + sum1;
+                        has_o = true;
+                    } else {
 #pragma unroll
-                    for (int c = 8; c < NCOL; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sraw[c]));
-                    tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                        for (int c = 0; c < NCOL / 2; ++c) pd[c] = 0u;
+                    }
+                    if (PAIR) {
+                        // block-diagonal P: this row weighs only its own half's tokens, the other 32 columns are zero
+                        uint32_t zero[32];
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) zero[c] = 0u;
+                        tmem_st32(lane_addr + COL_P + half * 32, pd);
+                        tmem_st32(lane_addr + COL_P + (half ^ 1) * 32, zero);
+                    } else {
+                        tmem_st32(lane_addr + COL_P, pd);
+                        tmem_st32(lane_addr + COL_P + 32, pd + (NCOL / 2 - 32));
+                    }
+                    bool fail = false;
+                    if (tok0 + STEP > total) {
+                        // last step of the sequence: V rows past the last key may hold anything, and they meet
+                        // weight-0 columns of P in the product: clear them (thread r clears row r of the stage)
+                        const int sv = it % NSV;
+                        fail = !mbar_wait(bar(B_VFULL + sv), (it / NSV) & 1, abort_flag);
+                        if (!fail && tok0 + tl >= total) {
+                            unsigned char* vrow = sm + SMEM_V + sv * STAGE_BYTES + tl * 128;
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                *reinterpret_cast<uint4*>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
+                                *reinterpret_cast<uint4*>(vrow + HALF_BYTES + c * 16) = make_uint4(0, 0, 0, 0);
+                            }
+                        }
+                        fence_async_smem();
+                    }
+                    tmem_wait_st();
+                    if (__any_sync(0xffffffffu, fail)) { ok = false; break; }
+                    if (tid == 64) TRACE(2, it, 5);
+                    tc_fence_before();
+                    mbar_arrive(bar(B_PFULL));
+                    if (tid == 64) TRACE(2, it, 6);
                 }
-                // move the reference maximum only when the tile exceeds it by more than the gap
-                float alpha = 1.f;
-                bool rescale = false;
-                if (valid && tmax > m_ref + kRescaleGap) {          // also true on the first finite tile (m_ref = -inf)
-                    alpha = exp2f(m_ref - tmax);                     // 0 when m_ref = -inf
-                    m_ref = tmax;
-                    l_run *= alpha;
-                    rescale = has_o;
+                if (!ok) break;
+
+                // ---- segment epilogue: wait for the last product, (PAIR) merge the two halves, write out ----
+                TRACE_MISC(5);
+                ok = mbar_wait_warp(bar(B_PVDONE), (it - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                TRACE_MISC(6);
+                float w_me = has_o ? 1.f : 0.f, w_other = 0.f, m_all = has_o ? m_ref : -INFINITY, l_all = l_run;
+                if (PAIR) {
+                    if (half == 1) {
+                        // hand the raw accumulator and the statistics to the lane that owns the row
+                        if (seg > 0) ok = mbar_wait(bar(B_XFREE), (seg - 1) & 1, abort_flag);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        xst[lrow] = make_float2(m_all, l_run);
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t o[32];
+                            tmem_ld32(lane_addr + COL_O + ch * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c4 = 0; c4 < 8; ++c4)
+                                xch[(ch * 8 + c4) * 64 + lrow] = make_float4(__uint_as_float(o[4 * c4]), __uint_as_float(o[4 * c4 + 1]),
+                                                                            __uint_as_float(o[4 * c4 + 2]), __uint_as_float(o[4 * c4 + 3]));
+                        }
+                        tc_fence_before();
+                        mbar_arrive(bar(B_XCH));
+                    } else {
+                        ok = mbar_wait_warp(bar(B_XCH), seg & 1, abort_flag);
+                        if (!ok) break;
+                        const float2 other = xst[lrow];
+                        m_all = fmaxf(m_all, other.x);
+                        const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
+                        w_me = has_o ? exp2f(m_ref - m_fin) : 0.f;
+                        w_other = exp2f(other.x - m_fin);               // 0 when the other half saw nothing
+                        l_all = l_run * w_me + other.y * w_other;
+                    }
                 }
-                if (__any_sync(0xffffffffu, rescale)) {
-                    // O was last written by the PV product of step t-1
-                    if (!mbar_wait_warp(bar(B_PVDONE + (bs ^ 1)), ((t - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
+                if (half == 0) {
+                    const bool final_out = sg.slot < 0;
+                    const float inv = final_out ? (l_all > 0.f ? 1.f / l_all : 0.f) : 1.f;
+                    __nv_bfloat16* orow = p.out + (((size_t)sg.b * N + node) * p.Hq + head) * D;
+                    float4* prow = p.part_o + (size_t)(final_out ? 0 : sg.slot) * 32 * ROWS + lrow;
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
                         uint32_t o[32];
                         tmem_ld32(lane_addr + COL_O + ch * 32, o);
                         tmem_wait_ld();
+                        float v[32];
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        tmem_st32(lane_addr + COL_O + ch * 32, o);
-                    }
-                }
-                if (tid == 64) TRACE(2, t, 3);
-                // P = exp2(x - m_ref) as bf16 pairs into the first 64 columns of S[bs] (column c holds tokens 2c, 2c+1)
-                uint32_t pd[NCOL / 2];
-                if (valid) {
-                    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                    float sum0 = 0.f, sum1 = 0.f;
+                        for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(o[c]) * w_me;
+                        if (PAIR) {
 #pragma unroll
-                    for (int c = 0; c < NCOL / 2; ++c) {
-                        const float e0 = exp2f(__uint_as_float(sraw[2 * c]) - m_use);
-                        const float e1 = exp2f(__uint_as_float(sraw[2 * c + 1]) - m_use);
-                        sum0 += e0; sum1 += e1;
-                        pd[c] = pack_bf16(e0, e1);
-                    }
-                    l_run += sum0 + sum1;
-                    has_o = true;
-                } else {
-#pragma unroll
-                    for (int c = 0; c < NCOL / 2; ++c) pd[c] = 0u;
-                }
-                uint32_t pk[64];
-                if (PAIR) {
-                    // block-diagonal P: this row weighs only its own half's tokens, the other 32 columns are zero
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) { pk[c] = half ? 0u : pd[c]; pk[32 + c] = half ? pd[c] : 0u; }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) pk[c] = pd[c % (NCOL / 2)];
-                }
-                tmem_st32(lane_addr + COL_S + bs * 128, pk);
-                tmem_st32(lane_addr + COL_S + bs * 128 + 32, pk + 32);
-                bool fail = false;
-                if (tok_begin + (t + 1) * STEP > total) {
-                    // last step of the sequence: V rows past the last key may hold anything, and they meet
-                    // weight-0 columns of P in the product: clear them (thread r clears row r of the stage)
-                    const int sv = t % NSV;
-                    fail = !mbar_wait(bar(B_VFULL + sv), (t / NSV) & 1, abort_flag);
-                    if (!fail && tok_begin + t * STEP + tl >= total) {
-                        unsigned char* vrow = sm + SMEM_V + sv * STAGE_BYTES + tl * 128;
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            *reinterpret_cast<uint4*>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
-                            *reinterpret_cast<uint4*>(vrow + HALF_BYTES + c * 16) = make_uint4(0, 0, 0, 0);
+                            for (int c4 = 0; c4 < 8; ++c4) {
+                                const float4 w = xch[(ch * 8 + c4) * 64 + lrow];
+                                v[4 * c4] += w.x * w_other; v[4 * c4 + 1] += w.y * w_other;
+                                v[4 * c4 + 2] += w.z * w_other; v[4 * c4 + 3] += w.w * w_other;
+                            }
                         }
-                    }
-                    fence_async_smem();
-                }
-                tmem_wait_st();
-                if (__any_sync(0xffffffffu, fail)) { ok = false; break; }
-                if (tid == 64) TRACE(2, t, 5);
-                tc_fence_before();
-                mbar_arrive(bar(B_PFULL + bs));
-                if (tid == 64) TRACE(2, t, 6);
-            }
-            // ---- epilogue: wait for the last product, (PAIR) merge the two halves, write out ----
-            TRACE_MISC(5);
-            if (ok) ok = mbar_wait_warp(bar(B_PVDONE + ((nsteps - 1) & 1)), ((nsteps - 1) >> 1) & 1, abort_flag);
-            TRACE_MISC(6);
-            // The rings are idle now (all copies landed, every product that read them has completed), so the
-            // K ring serves as the PAIR exchange area: [32 col4][64 rows] float4 (32 KB) followed by 64 float2.
-            float4* xch = reinterpret_cast<float4*>(sm + SMEM_K);
-            float2* xst = reinterpret_cast<float2*>(sm + SMEM_K + 32 * 64 * 16);
-            float w_me = 1.f, m_all = m_ref, l_all = l_run;
-            if (PAIR && ok) {
-                // lanes 64-127 hand their statistics to lanes 0-63, which answer with the merge weight
-                if (half == 1) {
-                    xst[lrow] = make_float2(has_o ? m_ref : -INFINITY, l_run);
-                    mbar_arrive(bar(B_XSTAT));
-                    ok = mbar_wait(bar(B_XWGT), 0, abort_flag);
-                    w_me = has_o ? xst[lrow].x : 0.f;
-                } else {
-                    ok = mbar_wait(bar(B_XSTAT), 0, abort_flag);
-                    const float2 other = xst[lrow];
-                    const float mm = has_o ? m_ref : -INFINITY;
-                    m_all = fmaxf(mm, other.x);
-                    const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
-                    w_me = has_o ? exp2f(m_ref - m_fin) : 0.f;
-                    const float w_other = exp2f(other.x - m_fin);       // 0 when the other half saw nothing
-                    l_all = l_run * w_me + other.y * w_other;
-                    xst[lrow] = make_float2(w_other, 0.f);
-                    mbar_arrive(bar(B_XWGT));
-                }
-                ok = __all_sync(0xffffffffu, ok);
-            }
-            TRACE_MISC(7);
-            if (ok) {
-                tc_fence_after();
-                const bool final_out = (p.n_split == 1);
-                const float inv = final_out ? (l_all > 0.f ? 1.f / l_all : 0.f) : 1.f;
-                const size_t slot = ((size_t)unit * p.n_split + split) * ROWS + lrow;
-                __nv_bfloat16* orow = p.out + (((size_t)b * N + node) * p.Hq + head) * D;
-                float* prow = p.part_o + slot * D;
+                        if (row_ok) {
+                            if (final_out) {
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t o[32];
-                    tmem_ld32(lane_addr + COL_O + ch * 32, o);
-                    tmem_wait_ld();
-                    float v[32];
+                                for (int c8 = 0; c8 < 4; ++c8)
+                                    *reinterpret_cast<uint4*>(orow + ch * 32 + c8 * 8) =
+                                        make_uint4(pack_bf16(v[8 * c8] * inv, v[8 * c8 + 1] * inv), pack_bf16(v[8 * c8 + 2] * inv, v[8 * c8 + 3] * inv),
+                                                   pack_bf16(v[8 * c8 + 4] * inv, v[8 * c8 + 5] * inv), pack_bf16(v[8 * c8 + 6] * inv, v[8 * c8 + 7] * inv));
+                            } else {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] = has_o ? __uint_as_float(o[c]) * w_me : 0.f;
-                    bool got = true;
-                    if (PAIR) {
-                        if (half == 1) {
-#pragma unroll
-                            for (int c4 = 0; c4 < 8; ++c4)
-                                xch[(ch * 8 + c4) * 64 + lrow] = make_float4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
-                            mbar_arrive(bar(B_XCH + ch));
-                        } else {
-                            got = mbar_wait(bar(B_XCH + ch), 0, abort_flag);
-                            if (got) {
-#pragma unroll
-                                for (int c4 = 0; c4 < 8; ++c4) {
-                                    const float4 w = xch[(ch * 8 + c4) * 64 + lrow];
-                                    v[4 * c4] += w.x; v[4 * c4 + 1] += w.y; v[4 * c4 + 2] += w.z; v[4 * c4 + 3] += w.w;
-                                }
+                                for (int c4 = 0; c4 < 8; ++c4)
+                                    prow[(size_t)(ch * 8 + c4) * ROWS] = make_float4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
                             }
                         }
                     }
-                    if (row_ok && half == 0 && got) {
+                    if (row_ok) {
                         if (final_out) {
-#pragma unroll
-                            for (int c8 = 0; c8 < 4; ++c8)
-                                *reinterpret_cast<uint4*>(orow + ch * 32 + c8 * 8) =
-                                    make_uint4(pack_bf16(v[8 * c8] * inv, v[8 * c8 + 1] * inv), pack_bf16(v[8 * c8 + 2] * inv, v[8 * c8 + 3] * inv),
-                                               pack_bf16(v[8 * c8 + 4] * inv, v[8 * c8 + 5] * inv), pack_bf16(v[8 * c8 + 6] * inv, v[8 * c8 + 7] * inv));
+                            if (p.lse) p.lse[((size_t)sg.b * p.Hq + head) * N + node] =
+                                l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
                         } else {
-#pragma unroll
-                            for (int c4 = 0; c4 < 8; ++c4)
-                                *reinterpret_cast<float4*>(prow + ch * 32 + c4 * 4) = make_float4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
+                            p.part_ml[(size_t)sg.slot * ROWS + lrow] = make_float2(l_all > 0.f ? m_all : -INFINITY, l_all);
                         }
                     }
+                    if (PAIR) mbar_arrive(bar(B_XFREE));
                 }
-                if (row_ok && half == 0) {
-                    if (final_out) {
-                        if (p.lse) p.lse[((size_t)b * p.Hq + head) * N + node] =
-                            l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
-                    } else {
-                        *reinterpret_cast<float2*>(p.part_ml + slot * 2) = make_float2(l_all > 0.f ? m_all : -INFINITY, l_all);
-                    }
-                }
-                tc_fence_before();
-            }
-        }
-    } else if (p.n_split > 1 || total == 0) {
-        // nothing to attend to in this range: an empty partial, or a zero output for an empty / rejected sequence
-        for (int idx = tid; idx < ROWS * (D / 4); idx += kThreads) {
-            const int r = idx / (D / 4), c4 = idx % (D / 4);
-            const int gr = mblock * 128 + r;
-            if (gr >= rows_total) continue;
-            if (p.n_split > 1) {
-                const size_t slot = ((size_t)unit * p.n_split + split) * ROWS + r;
-                *reinterpret_cast<float4*>(p.part_o + slot * D + c4 * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + slot * 2) = make_float2(-INFINITY, 0.f);
-            } else {
-                const int i = gr / G, hd = kvh * G + gr % G;
-                *reinterpret_cast<uint2*>(p.out + (((size_t)b * N + i) * p.Hq + hd) * D + c4 * 4) = make_uint2(0, 0);
-                if (c4 == 0 && p.lse) p.lse[((size_t)b * p.Hq + hd) * N + i] = -INFINITY;
+                tc_fence_before();        // the next segment's first product overwrites O
+                TRACE_MISC(7);
+                ++seg;
             }
         }
     }
 
     // ---- tear-down: everyone meets, TMEM goes back ----
     TRACE_MISC(8);
+    tc_fence_before();
     __syncthreads();
     TRACE_MISC(9);
-    if (nsteps > 0) {
-        if (warp == 1) {
-            tc_fence_after();
-            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
-        }
-        if (tid == 0 && *abort_flag) atomicCAS(p.status, 0, (int)VISPEC_E_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
     }
+    if (tid == 0 && *abort_flag) atomicCAS(p.status, 0, (int)VISPEC_E_TIMEOUT);
+    TL_END(p.trace_idx, 1);
+    CTA_T(1);
+}
+
+// Merge of the partials of every unit that more than one CTA worked on.  Grid (unit, group of 32 rows),
+// 8 warps; lane <-> row, warp w sums output columns 16w..16w+15 over the unit's segments.
+template <int ROWS>
+__global__ void __launch_bounds__(256)
+attn_tc5_merge_kernel(const Tc5Params p) {
+    __shared__ Sched sched;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    TL_START(p.trace_idx, 2);
+    pdl_launch_dependents();
+    if (warp == 0) sched_build(sched, p, lane);        // kv_len only: not written by the attention kernel
+    __syncthreads();
+    pdl_wait();                                        // the partials are complete
+    TL_START(p.trace_idx, 3);
+    const int upb = p.Hkv * p.n_mblocks;
+    const int unit = blockIdx.x, b = unit / upb, uib = unit - b * upb;
+    const int steps = sched.steps[b];
+    if (steps == 0) return;
+    const int T = sched.base[p.B];
+    const int geff = sched_ctas(T, sched.units, p.grid_attn, p.min_steps);
+    const int ub = sched.base[b] + uib * steps, ue = ub + steps;
+    const int c0 = cta_of(ub, T, geff), c1 = cta_of(ue - 1, T, geff);
+    if (c0 == c1) return;                              // one CTA had the whole unit and wrote the output itself
+    const int G = p.Hq / p.Hkv, N = p.N;
+    const int kvh = uib / p.n_mblocks, mblock = uib - kvh * p.n_mblocks;
+    const int lrow = blockIdx.y * 32 + lane;
+    const int row = mblock * 128 + lrow;
+    if (row >= G * N) return;
+    const int node = row / G, head = kvh * G + row % G;
+
+    auto slot_of = [&](int c) { return cta_lo(c, T, geff) >= ub ? 2 * c : 2 * c + 1; };
+    float m_all = -INFINITY;
+    for (int c = c0; c <= c1; ++c) m_all = fmaxf(m_all, __ldcg(&p.part_ml[(size_t)slot_of(c) * ROWS + lrow]).x);
+    const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
+    float l_all = 0.f;
+    float4 acc[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+    for (int c = c0; c <= c1; ++c) {
+        const int slot = slot_of(c);
+        const float2 ml = __ldcg(&p.part_ml[(size_t)slot * ROWS + lrow]);
+        const float w = exp2f(ml.x - m_fin);             // 0 for a segment that saw nothing
+        l_all += ml.y * w;
+        const float4* src = p.part_o + ((size_t)slot * 32 + warp * 4) * ROWS + lrow;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float4 v = __ldcg(src + (size_t)k * ROWS);
+            acc[k].x += w * v.x; acc[k].y += w * v.y; acc[k].z += w * v.z; acc[k].w += w * v.w;
+        }
+    }
+    const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+    __nv_bfloat16* orow = p.out + (((size_t)b * N + node) * p.Hq + head) * D + warp * 16;
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+        *reinterpret_cast<uint4*>(orow + k * 8) =
+            make_uint4(pack_bf16(acc[2 * k].x * inv, acc[2 * k].y * inv), pack_bf16(acc[2 * k].z * inv, acc[2 * k].w * inv),
+                       pack_bf16(acc[2 * k + 1].x * inv, acc[2 * k + 1].y * inv), pack_bf16(acc[2 * k + 1].z * inv, acc[2 * k + 1].w * inv));
+    if (p.lse && warp == 0)
+        p.lse[((size_t)b * p.Hq + head) * N + node] = l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 }  // namespace
@@ -592,10 +844,35 @@ extern "C" int vispec_debug_read_trace(long long* host) {
 extern "C" int vispec_debug_read_trace_misc(long long* host) {
     return cudaMemcpyFromSymbol(host, g_trace_misc, sizeof(g_trace_misc)) == cudaSuccess ? 0 : -1;
 }
+extern "C" int vispec_debug_cta_times(unsigned long long* host) {
+    return cudaMemcpyFromSymbol(host, g_cta_times, sizeof(g_cta_times)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int vispec_debug_set_trace_cta(int cta) {
+    return cudaMemcpyToSymbol(g_trace_cta, &cta, sizeof(int)) == cudaSuccess ? 0 : -1;
+}
+static int g_trace_launch = 0;
+extern "C" int vispec_debug_timeline(unsigned long long* host, int reset) {
+    if (reset) {
+        g_trace_launch = 0;
+        static unsigned long long init[4096][4];
+        for (int i = 0; i < 4096; ++i) { init[i][0] = ~0ull; init[i][1] = 0; init[i][2] = ~0ull; init[i][3] = ~0ull; }
+        return cudaMemcpyToSymbol(g_timeline, init, sizeof(init)) == cudaSuccess ? 0 : -1;
+    }
+    return cudaMemcpyFromSymbol(host, g_timeline, sizeof(g_timeline)) == cudaSuccess ? 0 : -1;
+}
 #endif
 
+static size_t tc5_partial_bytes(int grid, int rows) { return (size_t)2 * grid * rows * (D * 4 + 8); }
+
 bool attn_tc5_supports(const AttnArgs& a) {
-    return a.D == 128 && a.k_map && a.v_map && a.B > 0;
+    if (!(a.D == 128 && a.k_map && a.v_map && a.B > 0 && a.B <= kMaxB)) return false;
+    const int rows_total = (a.Hq / a.Hkv) * a.N;
+    const int rows = rows_total <= 64 ? 64 : 128;
+    const long long n_mblocks = rows_total <= 64 ? 1 : (rows_total + 127) / 128;
+    const long long t_max = (long long)a.B * a.Hkv * n_mblocks * ((a.S_max + STEP - 1) / STEP);
+    if (t_max * a.sm_count >= (1ll << 31)) return false;
+    if (!(a.scale > 0.f)) return false;       // the kernel takes the maximum before scaling
+    return kCounterBytes + tc5_partial_bytes(a.sm_count, rows) <= a.ws_bytes;
 }
 
 cudaError_t init_attn_tc5() {
@@ -611,33 +888,32 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     const int rows = pair ? 64 : 128;
     const int n_mblocks = pair ? 1 : (rows_total + 127) / 128;
     const int units = a.B * a.Hkv * n_mblocks;
-    const int max_steps = (a.S_max + STEP - 1) / STEP;
-    int n_split = a.sm_count / units;
-    if (n_split < 1) n_split = 1;
-    if (n_split > max_steps) n_split = max_steps;
-    const size_t part_bytes = (size_t)rows * (a.D * 4 + 8);
-    while (n_split > 1 && kCounterBytes + (size_t)units * n_split * part_bytes > a.ws_bytes) --n_split;
+    const long long t_max = (long long)units * ((a.S_max + STEP - 1) / STEP);
+    const int grid = (int)(t_max < a.sm_count ? t_max : a.sm_count);
 
     Tc5Params p;
     p.q = (const __nv_bfloat16*)a.q; p.kv_len = a.kv_len; p.mask = a.mask;
     p.out = (__nv_bfloat16*)a.out; p.lse = a.lse;
     unsigned char* ws = (unsigned char*)a.ws + kCounterBytes;
-    p.part_o = (float*)ws;
-    p.part_ml = (float*)(ws + (size_t)units * n_split * rows * a.D * 4);
-    p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_max = a.S_max; p.n_split = n_split; p.n_mblocks = n_mblocks;
+    p.part_o = (float4*)ws;
+    p.part_ml = (float2*)(ws + (size_t)2 * grid * rows * D * 4);
+    p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_max = a.S_max; p.n_mblocks = n_mblocks;
+    p.grid_attn = grid; p.min_steps = 2; p.early = a.early_prefetch ? 1 : 0;
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.status = a.status;
-    dim3 grid(n_split, units);
-    if (pair) attn_tc5_kernel<true><<<grid, kThreads, SMEM_ALLOC, st>>>(*a.k_map, *a.v_map, p);
-    else attn_tc5_kernel<false><<<grid, kThreads, SMEM_ALLOC, st>>>(*a.k_map, *a.v_map, p);
-    cudaError_t err = cudaGetLastError();
+#ifdef VISPEC_TC5_TRACE
+    p.trace_idx = g_trace_launch++;
+#else
+    p.trace_idx = 0;
+#endif
+    cudaError_t err = pair ? launch_pdl(attn_tc5_kernel<true>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, *a.k_map, *a.v_map, p)
+                           : launch_pdl(attn_tc5_kernel<false>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, *a.k_map, *a.v_map, p);
     if (err != cudaSuccess) return err;
     ++*n_launches;
-    if (n_split > 1) {
-        err = launch_attn_combine(a, n_split, n_mblocks, rows, st);
-        if (err != cudaSuccess) return err;
-        ++*n_launches;
-    }
+    err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 2), dim3(256), 0, st, p)
+               : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 4), dim3(256), 0, st, p);
+    if (err != cudaSuccess) return err;
+    ++*n_launches;
     return cudaSuccess;
 }
 

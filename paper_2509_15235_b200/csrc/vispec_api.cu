@@ -120,6 +120,15 @@ int vispec_ctx_set_workspace(vispec_ctx* c, void* ws, size_t bytes) {
     return VISPEC_OK;
 }
 
+int vispec_ctx_set_option(vispec_ctx* c, int option, int value) {
+    if (!c) return VISPEC_E_NULL;
+    switch (option) {
+        case VISPEC_OPT_EARLY_PREFETCH: c->early_prefetch = value != 0; return VISPEC_OK;
+        case VISPEC_OPT_FORCE_GENERIC: c->force_generic = value != 0; return VISPEC_OK;
+        default: return VISPEC_E_UNSUPPORTED;
+    }
+}
+
 int vispec_cache_register(vispec_ctx* c, int layer, void* k_cache, void* v_cache) {
     if (!c || !k_cache || !v_cache) return VISPEC_E_NULL;
     if (layer < 0 || layer >= c->shape.layers) return VISPEC_E_RANGE;
@@ -179,6 +188,7 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
     a.B = B; a.N = N; a.Hq = s.Hq; a.Hkv = s.Hkv; a.D = s.D; a.S_max = s.S_max;
     a.scale = scale; a.ws = c->ws; a.ws_bytes = c->ws_bytes; a.status = c->d_status;
     a.sm_count = c->sm_count;
+    a.early_prefetch = c->early_prefetch;
     a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
     int n = 0;
     cudaError_t err = (!c->force_generic && attn_tc5_supports(a)) ? launch_attn_tc5(a, (cudaStream_t)stream, &n)

@@ -19,7 +19,8 @@ struct vispec_ctx {
     void* ws = nullptr;             // caller-owned workspace
     size_t ws_bytes = 0;
     uint64_t launches = 0;
-    bool force_generic = false;     // VISPEC_FORCE_GENERIC=1 at context creation: debugging aid
+    bool force_generic = false;     // VISPEC_OPT_FORCE_GENERIC (or VISPEC_FORCE_GENERIC=1 at context creation)
+    bool early_prefetch = true;     // VISPEC_OPT_EARLY_PREFETCH
 };
 
 namespace vispec {
@@ -52,13 +53,14 @@ struct AttnArgs {
     void* ws; size_t ws_bytes;
     int* status;
     int sm_count;
+    bool early_prefetch;   // committed-prefix tiles may be read before the preceding kernel has completed
     const CUtensorMap* k_map; const CUtensorMap* v_map;
 };
 // Generic split-KV kernel on warp-level tensor-core instructions (any supported shape).
 cudaError_t init_attn_generic();   // once per device, with that device current
 cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, int* n_launches);
 
-// TMA + tcgen05 kernel (D = 128, G*N <= 64 query rows per kv head).
+// TMA + tcgen05 kernel (D = 128), work split evenly over the SMs, followed by its merge kernel.
 bool attn_tc5_supports(const AttnArgs& a);
 cudaError_t init_attn_tc5();           // once per device, with that device current
 cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches);
