@@ -103,11 +103,16 @@ typedef enum vispec_option {
     VISPEC_OPT_EARLY_PREFETCH = 1,
     /* Default 0 (1 if the environment has VISPEC_FORCE_GENERIC=1 at context creation).  Route attention
      * through the shape-generic warp-level kernel even where the TMA/tcgen05 kernel applies. */
-    VISPEC_OPT_FORCE_GENERIC = 2
+    VISPEC_OPT_FORCE_GENERIC = 2,
+    /* Default 0.  How the TMA/tcgen05 attention kernel combines the pieces of a (sequence, kv head) that
+     * several thread blocks work on: 0 chooses per call; 1 always parks partial results in the workspace
+     * and merges them with a second kernel; 2 uses thread-block clusters that merge through distributed
+     * shared memory whenever the shape allows one cluster per (sequence, kv head, row block). */
+    VISPEC_OPT_SPLIT_FORM = 3
 } vispec_option;
 
 /* Set an option of the context (host call, takes effect for later calls).  Errors: E_NULL,
- * E_UNSUPPORTED (unknown option). */
+ * E_UNSUPPORTED (unknown option), E_RANGE (value). */
 int vispec_ctx_set_option(vispec_ctx* ctx, int option, int value);
 
 /* Register layer `layer`'s cache pair [B_max,Hkv,S_max,D] bf16 (App. A: pre-allocated KV cache).

@@ -29,6 +29,7 @@ EXPORTS = [
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
+OPT_SPLIT_FORM = 3
 
 
 class VispecShape(ctypes.Structure):

@@ -77,6 +77,7 @@ extern "C" int vispec_tree_verify_attn_static(const void* q, const void* k_cache
     a.status = status_word ? status_word : s.status;
     a.sm_count = s.sm_count;
     a.early_prefetch = false;
+    a.tc5_path = 0;
     a.k_map = nullptr; a.v_map = nullptr;
     int n = 0;
     return vispec::launch_attn_generic(a, (cudaStream_t)stream, &n) == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;

@@ -19,10 +19,11 @@
 //   warp 1     tensor-core issuer (one thread): S = Q K^T and O += P V as 128x128x16 tcgen05.mma, owns TMEM
 //   warps 2-5  softmax: thread <-> TMEM lane, i.e. one thread per accumulator row, no shuffles; they also
 //              load Q at the start of every segment and run the segment epilogue
-// TMEM map (512 columns x 128 lanes): S[0] 0..127, S[1] 128..255, O 256..383, Q 384..447, P 448..511.
-// Q and P (bf16, packed two per column) are the A operands of the S and PV products, so neither ever
-// touches shared memory.  S is double-buffered and released as soon as the softmax threads have read it,
-// so the S product of step u+1 runs while step u is in the softmax.
+// TMEM map (512 columns x 128 lanes): S[0] 0..127, S[1] 128..255, O 256..383, P[0] 384..447, P[1] 448..511.
+// P (bf16, packed two per column) is the A operand of the PV product and never touches shared memory; Q
+// sits in shared memory in the same swizzled K-major layout as a K stage.  S and P are double-buffered: S
+// is released as soon as the softmax threads have read it, so the S product of step u+1 and the PV
+// product of step u-1 run while step u is in the softmax.
 //
 // Two row layouts share the code:
 //   FULL  (G*N > 64):  lane r holds query row r of the block; a thread handles all 128 tokens of a step.
@@ -56,19 +57,21 @@ constexpr int kThreads = 192;
 constexpr int kMaxB = 64;                      // sequences per call this kernel takes
 constexpr int SMEM_K = 0;
 constexpr int SMEM_V = SMEM_K + NSK * STAGE_BYTES;
-constexpr int SMEM_X = SMEM_V + NSV * STAGE_BYTES;             // PAIR exchange: [32 col4][64 rows] float4 + 64 float2
-constexpr int X_BYTES = 32 * 64 * 16 + 64 * 8;
-constexpr int SMEM_BAR = SMEM_X + X_BYTES;
+constexpr int SMEM_Q = SMEM_V + NSV * STAGE_BYTES;             // Q tile, 128 rows, laid out like a K stage; between
+                                                               // segments it is the PAIR exchange [32 col4][64 rows] float4
+constexpr int SMEM_XST = SMEM_Q + STAGE_BYTES;                 // PAIR exchange of statistics: 64 float2
+constexpr int SMEM_BAR = SMEM_XST + 64 * 8;
 constexpr int BAR_BYTES = 256;
 constexpr int SMEM_SCHED = SMEM_BAR + BAR_BYTES;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t COL_S = 0, COL_O = 256, COL_Q = 384, COL_P = 448;
+constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384;
 constexpr float kRescaleGap = 8.0f;                            // log2 units
 constexpr long long kWaitCycles = 1500000000LL;                // ~0.8 s at 1.9 GHz
 
 enum { B_KFULL = 0, B_KEMPTY = B_KFULL + NSK, B_VFULL = B_KEMPTY + NSK, B_VEMPTY = B_VFULL + NSV,
-       B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 1,
-       B_QFULL = B_PVDONE + 1, B_XCH = B_QFULL + 1, B_XFREE = B_XCH + 1, B_COUNT = B_XFREE + 1 };
+       B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2,
+       B_QFULL = B_PVDONE + 2, B_XCH = B_QFULL + 1, B_XFREE = B_XCH + 1,
+       B_EPI = B_XFREE + 1, B_CL1 = B_EPI + 1, B_COUNT = B_CL1 + 1 };
 static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block too small");
 
 // The schedule every CTA (and the merge kernel) derives from kv_len.
@@ -130,6 +133,44 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// Thread-block cluster helpers (distributed shared memory).
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank)); return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ float4 dsmem_ld4(uint32_t a) {
+    float4 v; asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory"); return v;
+}
+__device__ __forceinline__ float2 dsmem_ld2(uint32_t a) {
+    float2 v; asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a) : "memory"); return v;
+}
+// Bounded wait like mbar_wait, acquiring at cluster scope (the arrivals come from other CTAs of the cluster).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 63) == 63) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+        }
+    }
+}
 // Programmatic dependent launch: let the next kernel in the stream be scheduled / wait for the previous one.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -143,6 +184,17 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
         "mov.b64 db, {%2, %3};\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The same with both operands described in shared memory.
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 // 32 lanes x 32 bit, 32 consecutive columns: thread i of the warp accesses lane (base lane + i).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
@@ -296,7 +348,15 @@ struct Seg {
 struct SegIter {
     const Sched* s;
     int B, n_mblocks, g, lo, hi, cta;
+    bool cl, cl_done;          // cluster schedule: exactly one segment (possibly empty), given in cl_seg
+    Seg cl_seg;
     __device__ __forceinline__ bool next(Seg& o) {
+        if (cl) {
+            if (cl_done) return false;
+            cl_done = true;
+            o = cl_seg;
+            return true;
+        }
         if (g >= hi) return false;
         int l = 0, r = B;                               // first b with base[b] > g, minus one
         while (l < r) { const int m = (l + r) >> 1; if (s->base[m] <= g) l = m + 1; else r = m; }
@@ -316,7 +376,7 @@ struct SegIter {
     }
 };
 
-template <bool PAIR>
+template <bool PAIR, bool CL>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const Tc5Params p) {
     constexpr int ROWS = PAIR ? 64 : 128;      // distinct query rows per CTA
@@ -344,9 +404,12 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         for (int i = 0; i < NSV; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(B_SFULL + i), 1); mbar_init(bar(B_SFREE + i), 128);
+            mbar_init(bar(B_PFULL + i), 128); mbar_init(bar(B_PVDONE + i), 1);
         }
-        mbar_init(bar(B_PFULL), 128); mbar_init(bar(B_PVDONE), 1); mbar_init(bar(B_QFULL), 128);
+        mbar_init(bar(B_QFULL), 128);
         mbar_init(bar(B_XCH), 64); mbar_init(bar(B_XFREE), 64);
+        mbar_init(bar(B_EPI), 128);
+        mbar_init(bar(B_CL1), CL ? cluster_size() : 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -360,15 +423,34 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     TRACE_MISC(1);
     tc_fence_before();
     __syncthreads();
+    if (CL) cluster_sync_all();          // every CTA's barriers exist before a peer can signal them
     tc_fence_after();
     TRACE_MISC(2);
 
+    // Schedule.  Cluster form: cluster <-> unit, the CTA of rank r takes the r-th of k equal parts of the
+    // unit's steps (an empty part still takes part in the exchange).  Otherwise: equal ranges of the line of
+    // all steps.
     const int T = sched.base[p.B];
-    const int geff = T > 0 ? sched_ctas(T, sched.units, (int)gridDim.x, p.min_steps) : 0;
+    const int geff = CL ? (int)gridDim.x : (T > 0 ? sched_ctas(T, sched.units, (int)gridDim.x, p.min_steps) : 0);
     const bool active = cta < geff;
-    const int lo = active ? cta_lo(cta, T, geff) : 0, hi = active ? cta_lo(cta + 1, T, geff) : 0;
+    const int lo = (!CL && active) ? cta_lo(cta, T, geff) : 0, hi = (!CL && active) ? cta_lo(cta + 1, T, geff) : 0;
     const uint32_t tmem = *tmem_slot;
-    auto make_iter = [&]() { SegIter it; it.s = &sched; it.B = p.B; it.n_mblocks = p.n_mblocks; it.g = lo; it.lo = lo; it.hi = hi; it.cta = cta; return it; };
+    const int ck = CL ? (int)cluster_size() : 1, cr = CL ? (int)cluster_ctarank() : 0;
+    Seg cl_seg = {};
+    if (CL) {
+        const int upb = p.Hkv * p.n_mblocks;
+        const int unit = cta / ck, b = unit / upb, uib = unit - b * upb;
+        cl_seg.b = b; cl_seg.kvh = uib / p.n_mblocks; cl_seg.mblock = uib - cl_seg.kvh * p.n_mblocks;
+        cl_seg.steps = sched.steps[b]; cl_seg.S = sched.len[b];
+        cl_seg.st0 = (cr * cl_seg.steps) / ck;
+        cl_seg.n = ((cr + 1) * cl_seg.steps) / ck - cl_seg.st0;
+        cl_seg.slot = -1;
+    }
+    auto make_iter = [&]() {
+        SegIter it; it.s = &sched; it.B = p.B; it.n_mblocks = p.n_mblocks; it.g = lo; it.lo = lo; it.hi = hi; it.cta = cta;
+        it.cl = CL; it.cl_done = false; it.cl_seg = cl_seg;
+        return it;
+    };
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -414,9 +496,9 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             constexpr uint32_t IDESC_O = instr_desc(1);            // B = V stage, MN-major
             constexpr uint32_t DESC_HI = desc_hi(1024);            // 8 rows x 128 B between row groups, everywhere
             auto issue_pv = [&](int u, uint32_t acc) -> bool {
-                const int sv = u % NSV;
+                const int bu = u & 1, sv = u % NSV;
                 TRACE(1, u, 3);
-                if (!mbar_wait(bar(B_PFULL), u & 1, abort_flag)) return false;
+                if (!mbar_wait(bar(B_PFULL + bu), (u >> 1) & 1, abort_flag)) return false;
                 TRACE(1, u, 4);
                 if (!mbar_wait(bar(B_VFULL + sv), (u / NSV) & 1, abort_flag)) return false;
                 TRACE(1, u, 5);
@@ -424,10 +506,10 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 const uint32_t vb = desc_lo(base + SMEM_V + sv * STAGE_BYTES, HALF_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < STEP / 16; ++ks)      // 16 tokens per instruction: 8 P columns, 16 V rows (2 KB)
-                    tc_mma_ts(tmem + COL_O, tmem + COL_P + ks * 8, vb + ks * 128, DESC_HI, IDESC_O,
+                    tc_mma_ts(tmem + COL_O, tmem + COL_P + bu * 64 + ks * 8, vb + ks * 128, DESC_HI, IDESC_O,
                               (acc || ks > 0) ? 1u : 0u);
                 tc_commit(bar(B_VEMPTY + sv));
-                tc_commit(bar(B_PVDONE));
+                tc_commit(bar(B_PVDONE + bu));
                 TRACE(1, u, 6);
                 return true;
             };
@@ -450,10 +532,12 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     if (it >= 2 && !mbar_wait(bar(B_SFREE + bs), ((it >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t kb = desc_lo(base + SMEM_K + sk * STAGE_BYTES, 16);
+                    const uint32_t qb = desc_lo(base + SMEM_Q, 16);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)         // 16 d-columns per instruction: 8 Q columns, 32 B of each K row
-                        tc_mma_ts(tmem + COL_S + bs * 128, tmem + COL_Q + ks * 8,
-                                  kb + (((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4), DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+                    for (int ks = 0; ks < D / 16; ++ks) {       // 16 d-columns per instruction: 32 B of each Q and K row
+                        const uint32_t koff = ((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
+                        tc_mma_ss(tmem + COL_S + bs * 128, qb + koff, DESC_HI, kb + koff, DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+                    }
                     tc_commit(bar(B_KEMPTY + sk));
                     tc_commit(bar(B_SFULL + bs));
                     TRACE(1, it, 2);
@@ -492,27 +576,35 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             if (any_bad && cta == 0 && st == 0) atomicCAS(p.status, 0, (int)VISPEC_E_RANGE);
         }
 
-        // Q of a segment -> TMEM buffer `buf`: each thread packs its row (bf16 pairs) into 64 columns
-        auto load_q = [&](const Seg& sg) {
-            const int row = sg.mblock * 128 + lrow;
-            uint32_t qreg[64];
-            if (row < rows_total) {
-                const int node = row / G, head = sg.kvh * G + row % G;
-                const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)sg.b * N + node) * p.Hq + head) * D);
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const uint4 v4 = src[c];
-                    qreg[4 * c] = v4.x; qreg[4 * c + 1] = v4.y; qreg[4 * c + 2] = v4.z; qreg[4 * c + 3] = v4.w;
-                }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 64; ++c) qreg[c] = 0u;
+        // Q of a segment -> shared memory, rows in the swizzled K-major layout of a K stage (PAIR: rows 64-127
+        // repeat rows 0-63).  Thread t moves 16-byte chunk t%16 of rows t/16, t/16 + 8, ...
+        auto load_q = [&](const Seg& sg, int seg) -> bool {
+            if (PAIR && seg > 0) {
+                // the tile doubles as the exchange area of the previous segment's epilogue
+                if (!mbar_wait_warp(bar(B_XFREE), (seg - 1) & 1, abort_flag)) return false;
             }
-            tmem_st32(lane_addr + COL_Q, qreg);
-            tmem_st32(lane_addr + COL_Q + 32, qreg + 32);
-            tmem_wait_st();
-            tc_fence_before();
+            constexpr int ITEMS = ROWS * 16 / 128;
+            const int ch = st & 15;
+            uint4 v[ITEMS];
+#pragma unroll
+            for (int k = 0; k < ITEMS; ++k) {
+                const int row = sg.mblock * 128 + (st >> 4) + 8 * k;
+                v[k] = make_uint4(0, 0, 0, 0);
+                if (row < rows_total) {
+                    const int node = row / G, head = sg.kvh * G + row % G;
+                    v[k] = *(reinterpret_cast<const uint4*>(p.q + (((size_t)sg.b * N + node) * p.Hq + head) * D) + ch);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < ITEMS; ++k) {
+                const int r = (st >> 4) + 8 * k;
+                unsigned char* dst = sm + SMEM_Q + (ch >> 3) * HALF_BYTES + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
+                *reinterpret_cast<uint4*>(dst) = v[k];
+                if (PAIR) *reinterpret_cast<uint4*>(dst + 64 * 128) = v[k];
+            }
+            fence_async_smem();
             mbar_arrive(bar(B_QFULL));
+            return true;
         };
 
         if (active) {
@@ -520,11 +612,11 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             Seg sg;
             int it = 0, seg = 0;
             bool ok = true;
-            float4* xch = reinterpret_cast<float4*>(sm + SMEM_X);
-            float2* xst = reinterpret_cast<float2*>(sm + SMEM_X + 32 * 64 * 16);
+            float4* xch = reinterpret_cast<float4*>(sm + SMEM_Q);
+            float2* xst = reinterpret_cast<float2*>(sm + SMEM_XST);
             while (ok && si.next(sg)) {
                 // every S product of the previous segment has been consumed by now, so Q may be replaced
-                load_q(sg);
+                if (!load_q(sg, seg)) { ok = false; break; }
                 TRACE_MISC(3);
 
                 const int row = sg.mblock * 128 + lrow;          // query row within the kv head's G*N rows
@@ -589,12 +681,10 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                         l_run *= alpha;
                         rescale = has_o;
                     }
-                    // the PV product of step it-1 must be complete before P is replaced (and before O is touched)
-                    if (it >= 1) {
-                        if (!mbar_wait_warp(bar(B_PVDONE), (it - 1) & 1, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                    }
                     if (__any_sync(0xffffffffu, rescale)) {
+                        // O was last written by the PV product of step it-1 (same segment: has_o is set)
+                        if (!mbar_wait_warp(bar(B_PVDONE + (bs ^ 1)), ((it - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch) {
                             uint32_t o[32];
@@ -624,16 +714,21 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
 #pragma unroll
                         for (int c = 0; c < NCOL / 2; ++c) pd[c] = 0u;
                     }
+                    // P[bs] is free once the PV product of step it-2 has completed
+                    if (it >= 2) {
+                        if (!mbar_wait_warp(bar(B_PVDONE + bs), ((it >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                    }
                     if (PAIR) {
                         // block-diagonal P: this row weighs only its own half's tokens, the other 32 columns are zero
                         uint32_t zero[32];
 #pragma unroll
                         for (int c = 0; c < 32; ++c) zero[c] = 0u;
-                        tmem_st32(lane_addr + COL_P + half * 32, pd);
-                        tmem_st32(lane_addr + COL_P + (half ^ 1) * 32, zero);
+                        tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pd);
+                        tmem_st32(lane_addr + COL_P + bs * 64 + (half ^ 1) * 32, zero);
                     } else {
-                        tmem_st32(lane_addr + COL_P, pd);
-                        tmem_st32(lane_addr + COL_P + 32, pd + (NCOL / 2 - 32));
+                        tmem_st32(lane_addr + COL_P + bs * 64, pd);
+                        tmem_st32(lane_addr + COL_P + bs * 64 + 32, pd + (NCOL / 2 - 32));
                     }
                     bool fail = false;
                     if (tok0 + STEP > total) {
@@ -655,24 +750,22 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     if (__any_sync(0xffffffffu, fail)) { ok = false; break; }
                     if (tid == 64) TRACE(2, it, 5);
                     tc_fence_before();
-                    mbar_arrive(bar(B_PFULL));
+                    mbar_arrive(bar(B_PFULL + bs));
                     if (tid == 64) TRACE(2, it, 6);
                 }
                 if (!ok) break;
 
                 // ---- segment epilogue: wait for the last product, (PAIR) merge the two halves, write out ----
                 TRACE_MISC(5);
-                ok = mbar_wait_warp(bar(B_PVDONE), (it - 1) & 1, abort_flag);
+                if (sg.n > 0) ok = mbar_wait_warp(bar(B_PVDONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 TRACE_MISC(6);
                 float w_me = has_o ? 1.f : 0.f, w_other = 0.f, m_all = has_o ? m_ref : -INFINITY, l_all = l_run;
                 if (PAIR) {
                     if (half == 1) {
-                        // hand the raw accumulator and the statistics to the lane that owns the row
-                        if (seg > 0) ok = mbar_wait(bar(B_XFREE), (seg - 1) & 1, abort_flag);
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) break;
+                        // hand the raw accumulator and the statistics to the lane that owns the row (the Q tile
+                        // is idle: every S product of the segment has completed)
                         xst[lrow] = make_float2(m_all, l_run);
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch) {
@@ -697,11 +790,15 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                         l_all = l_run * w_me + other.y * w_other;
                     }
                 }
+                // O is only defined once a product has run (an empty cluster part never ran one): select, never
+                // multiply, where the weight is zero
+                float4* pbuf = reinterpret_cast<float4*>(sm + SMEM_K);                       // cluster form: [32 col4][ROWS]
+                float2* pst = reinterpret_cast<float2*>(sm + SMEM_K + 32 * ROWS * 16);       //               [ROWS] (m, l)
                 if (half == 0) {
-                    const bool final_out = sg.slot < 0;
+                    const bool final_out = !CL && sg.slot < 0;
                     const float inv = final_out ? (l_all > 0.f ? 1.f / l_all : 0.f) : 1.f;
                     __nv_bfloat16* orow = p.out + (((size_t)sg.b * N + node) * p.Hq + head) * D;
-                    float4* prow = p.part_o + (size_t)(final_out ? 0 : sg.slot) * 32 * ROWS + lrow;
+                    float4* prow = CL ? pbuf + lrow : p.part_o + (size_t)(final_out ? 0 : sg.slot) * 32 * ROWS + lrow;
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
                         uint32_t o[32];
@@ -709,38 +806,98 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                         tmem_wait_ld();
                         float v[32];
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(o[c]) * w_me;
+                        for (int c = 0; c < 32; ++c) v[c] = has_o ? __uint_as_float(o[c]) * w_me : 0.f;
                         if (PAIR) {
+                            if (w_other > 0.f) {
 #pragma unroll
-                            for (int c4 = 0; c4 < 8; ++c4) {
-                                const float4 w = xch[(ch * 8 + c4) * 64 + lrow];
-                                v[4 * c4] += w.x * w_other; v[4 * c4 + 1] += w.y * w_other;
-                                v[4 * c4 + 2] += w.z * w_other; v[4 * c4 + 3] += w.w * w_other;
+                                for (int c4 = 0; c4 < 8; ++c4) {
+                                    const float4 w = xch[(ch * 8 + c4) * 64 + lrow];
+                                    v[4 * c4] += w.x * w_other; v[4 * c4 + 1] += w.y * w_other;
+                                    v[4 * c4 + 2] += w.z * w_other; v[4 * c4 + 3] += w.w * w_other;
+                                }
                             }
                         }
-                        if (row_ok) {
-                            if (final_out) {
+                        if (final_out) {
+                            if (row_ok) {
 #pragma unroll
                                 for (int c8 = 0; c8 < 4; ++c8)
                                     *reinterpret_cast<uint4*>(orow + ch * 32 + c8 * 8) =
                                         make_uint4(pack_bf16(v[8 * c8] * inv, v[8 * c8 + 1] * inv), pack_bf16(v[8 * c8 + 2] * inv, v[8 * c8 + 3] * inv),
                                                    pack_bf16(v[8 * c8 + 4] * inv, v[8 * c8 + 5] * inv), pack_bf16(v[8 * c8 + 6] * inv, v[8 * c8 + 7] * inv));
-                            } else {
-#pragma unroll
-                                for (int c4 = 0; c4 < 8; ++c4)
-                                    prow[(size_t)(ch * 8 + c4) * ROWS] = make_float4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
                             }
+                        } else if (CL || row_ok) {
+#pragma unroll
+                            for (int c4 = 0; c4 < 8; ++c4)
+                                prow[(size_t)(ch * 8 + c4) * ROWS] = make_float4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
                         }
                     }
-                    if (row_ok) {
+                    const float2 stat = make_float2(l_all > 0.f ? m_all : -INFINITY, l_all);
+                    if (CL) {
+                        pst[lrow] = stat;
+                    } else if (row_ok) {
                         if (final_out) {
                             if (p.lse) p.lse[((size_t)sg.b * p.Hq + head) * N + node] =
                                 l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
                         } else {
-                            p.part_ml[(size_t)sg.slot * ROWS + lrow] = make_float2(l_all > 0.f ? m_all : -INFINITY, l_all);
+                            p.part_ml[(size_t)sg.slot * ROWS + lrow] = stat;
                         }
                     }
                     if (PAIR) mbar_arrive(bar(B_XFREE));
+                }
+                if (CL) {
+                    // ---- cluster exchange: every CTA of the unit has parked its partial in its own shared memory;
+                    // rank r merges rows [r*rp, (r+1)*rp) of all k partials and writes them out ----
+                    mbar_arrive(bar(B_EPI));
+                    bool eok = true;
+                    if (st == 0) {
+                        eok = mbar_wait(bar(B_EPI), 0, abort_flag);
+                        // signal every CTA of the cluster (this one included), whatever happened here: a peer
+                        // must never be left waiting
+                        for (int j = 0; j < ck; ++j) mbar_arrive_remote(dsmem_addr(bar(B_CL1), (uint32_t)j));
+                    }
+                    eok = mbar_wait_cluster(bar(B_CL1), 0, abort_flag) && eok;
+                    ok = __all_sync(0xffffffffu, eok);
+                    if (ok) {
+                        const int rp = (ROWS + ck - 1) / ck;
+                        const int row0 = cr * rp;
+                        const int nrows = min(rp, ROWS - row0);
+                        const uint32_t pbuf_a = base + SMEM_K, pst_a = base + SMEM_K + 32 * ROWS * 16;
+                        for (int item = st; item < nrows * 32; item += 128) {
+                            const int c4 = item / nrows, lr = row0 + (item - c4 * nrows);
+                            const int grow = sg.mblock * 128 + lr;
+                            if (grow >= rows_total) continue;
+                            float2 ml[8];
+                            float4 pv[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                ml[j] = make_float2(-INFINITY, 0.f);
+                                pv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (j < ck) {
+                                    ml[j] = dsmem_ld2(dsmem_addr(pst_a + lr * 8, (uint32_t)j));
+                                    pv[j] = dsmem_ld4(dsmem_addr(pbuf_a + (c4 * ROWS + lr) * 16, (uint32_t)j));
+                                }
+                            }
+                            float mm = -INFINITY;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) mm = fmaxf(mm, ml[j].x);
+                            const float m_fin = (mm == -INFINITY) ? 0.f : mm;
+                            float ll = 0.f;
+                            float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float w = exp2f(ml[j].x - m_fin);          // 0 for an empty or absent part
+                                ll += ml[j].y * w;
+                                a4.x += w * pv[j].x; a4.y += w * pv[j].y; a4.z += w * pv[j].z; a4.w += w * pv[j].w;
+                            }
+                            const float inv2 = ll > 0.f ? 1.f / ll : 0.f;
+                            const int nd = grow / G, hd = sg.kvh * G + grow % G;
+                            *reinterpret_cast<uint2*>(p.out + (((size_t)sg.b * N + nd) * p.Hq + hd) * D + c4 * 4) =
+                                make_uint2(pack_bf16(a4.x * inv2, a4.y * inv2), pack_bf16(a4.z * inv2, a4.w * inv2));
+                            if (c4 == 0 && p.lse)
+                                p.lse[((size_t)sg.b * p.Hq + hd) * N + nd] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
+                        }
+                    }
+                    if (!ok) break;
                 }
                 tc_fence_before();        // the next segment's first product overwrites O
                 TRACE_MISC(7);
@@ -753,6 +910,9 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     TRACE_MISC(8);
     tc_fence_before();
     __syncthreads();
+    // Cluster form: nobody leaves while a peer may still read its shared memory or signal its barriers.  Every
+    // CTA gets here (all its other waits are bounded), so this hardware barrier ends.
+    if (CL) cluster_sync_all();
     TRACE_MISC(9);
     if (warp == 1) {
         tc_fence_after();
@@ -763,75 +923,112 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     CTA_T(1);
 }
 
-// Merge of the partials of every unit that more than one CTA worked on.  Grid (unit, group of 32 rows),
-// 8 warps; lane <-> row, warp w sums output columns 16w..16w+15 over the unit's segments.
+// Merge of the partials of every unit that more than one CTA worked on.  Grid (unit, 2 * group of 32 rows +
+// half of the columns), 4 warps; lane <-> row, a warp sums 16 output columns over the unit's segments.
+// The blocks are small so that they fit beside a resident attention CTA: they are launched early
+// (programmatic dependent launch) and must not keep the next layer's attention CTAs off the SMs.
 template <int ROWS>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 attn_tc5_merge_kernel(const Tc5Params p) {
-    __shared__ Sched sched;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    TL_START(p.trace_idx, 2);
     pdl_launch_dependents();
-    if (warp == 0) sched_build(sched, p, lane);        // kv_len only: not written by the attention kernel
-    __syncthreads();
-    pdl_wait();                                        // the partials are complete
-    TL_START(p.trace_idx, 3);
+    // The schedule, recomputed per thread from kv_len (which the attention kernel does not write) without
+    // shared memory: beside a resident attention CTA an SM has no shared memory to spare.
     const int upb = p.Hkv * p.n_mblocks;
     const int unit = blockIdx.x, b = unit / upb, uib = unit - b * upb;
-    const int steps = sched.steps[b];
-    if (steps == 0) return;
-    const int T = sched.base[p.B];
-    const int geff = sched_ctas(T, sched.units, p.grid_attn, p.min_steps);
-    const int ub = sched.base[b] + uib * steps, ue = ub + steps;
+    int T = 0, live = 0, base_b = 0, steps = 0;
+    for (int bb = 0; bb < p.B; ++bb) {
+        const int S = p.kv_len[bb];
+        const int st = (S >= 0 && S + p.N <= p.S_max) ? (S + p.N + STEP - 1) / STEP : 0;
+        if (bb == b) { base_b = T; steps = st; }
+        T += st * upb;
+        live += st > 0 ? upb : 0;
+    }
+    pdl_wait();                                        // the partials are complete
+    TL_START(p.trace_idx, 3);
+    if (steps == 0) { TL_END(p.trace_idx, 2); return; }
+    const int geff = sched_ctas(T, live, p.grid_attn, p.min_steps);
+    const int ub = base_b + uib * steps, ue = ub + steps;
     const int c0 = cta_of(ub, T, geff), c1 = cta_of(ue - 1, T, geff);
-    if (c0 == c1) return;                              // one CTA had the whole unit and wrote the output itself
+    if (c0 == c1) { TL_END(p.trace_idx, 2); return; }                              // one CTA had the whole unit and wrote the output itself
     const int G = p.Hq / p.Hkv, N = p.N;
     const int kvh = uib / p.n_mblocks, mblock = uib - kvh * p.n_mblocks;
-    const int lrow = blockIdx.y * 32 + lane;
+    const int lrow = (blockIdx.y >> 1) * 32 + lane;
+    const int cw = (blockIdx.y & 1) * 4 + warp;         // which 16 output columns
     const int row = mblock * 128 + lrow;
-    if (row >= G * N) return;
+    if (row >= G * N) { TL_END(p.trace_idx, 2); return; }
     const int node = row / G, head = kvh * G + row % G;
 
     auto slot_of = [&](int c) { return cta_lo(c, T, geff) >= ub ? 2 * c : 2 * c + 1; };
-    float m_all = -INFINITY;
-    for (int c = c0; c <= c1; ++c) m_all = fmaxf(m_all, __ldcg(&p.part_ml[(size_t)slot_of(c) * ROWS + lrow]).x);
-    const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
-    float l_all = 0.f;
+    // Segments are taken four at a time with every load of a group issued before the first use, so that a
+    // group costs one memory round trip; groups are folded with the usual running-maximum rescale.
+    float m_all = -INFINITY, l_all = 0.f;
     float4 acc[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-    for (int c = c0; c <= c1; ++c) {
-        const int slot = slot_of(c);
-        const float2 ml = __ldcg(&p.part_ml[(size_t)slot * ROWS + lrow]);
-        const float w = exp2f(ml.x - m_fin);             // 0 for a segment that saw nothing
-        l_all += ml.y * w;
-        const float4* src = p.part_o + ((size_t)slot * 32 + warp * 4) * ROWS + lrow;
+    for (int cb = c0; cb <= c1; cb += 4) {
+        float2 ml[4];
+        float4 v[4][4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float4 v = __ldcg(src + (size_t)k * ROWS);
-            acc[k].x += w * v.x; acc[k].y += w * v.y; acc[k].z += w * v.z; acc[k].w += w * v.w;
+        for (int j = 0; j < 4; ++j) {
+            const int c = cb + j;
+            ml[j] = make_float2(-INFINITY, 0.f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v[j][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c <= c1) {
+                const int slot = slot_of(c);
+                ml[j] = __ldcg(&p.part_ml[(size_t)slot * ROWS + lrow]);
+                const float4* src = p.part_o + ((size_t)slot * 32 + cw * 4) * ROWS + lrow;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) v[j][k] = __ldcg(src + (size_t)k * ROWS);
+            }
         }
+        float m_new = m_all;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m_new = fmaxf(m_new, ml[j].x);
+        const float m_fin = (m_new == -INFINITY) ? 0.f : m_new;
+        const float a = exp2f(m_all - m_fin);                 // 0 while nothing has been accumulated
+        l_all *= a;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { acc[k].x *= a; acc[k].y *= a; acc[k].z *= a; acc[k].w *= a; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float w = exp2f(ml[j].x - m_fin);           // 0 for a segment that saw nothing (or is absent)
+            l_all += ml[j].y * w;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc[k].x += w * v[j][k].x; acc[k].y += w * v[j][k].y; acc[k].z += w * v[j][k].z; acc[k].w += w * v[j][k].w;
+            }
+        }
+        m_all = m_new;
     }
     const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
-    __nv_bfloat16* orow = p.out + (((size_t)b * N + node) * p.Hq + head) * D + warp * 16;
+    __nv_bfloat16* orow = p.out + (((size_t)b * N + node) * p.Hq + head) * D + cw * 16;
 #pragma unroll
     for (int k = 0; k < 2; ++k)
         *reinterpret_cast<uint4*>(orow + k * 8) =
             make_uint4(pack_bf16(acc[2 * k].x * inv, acc[2 * k].y * inv), pack_bf16(acc[2 * k].z * inv, acc[2 * k].w * inv),
                        pack_bf16(acc[2 * k + 1].x * inv, acc[2 * k + 1].y * inv), pack_bf16(acc[2 * k + 1].z * inv, acc[2 * k + 1].w * inv));
-    if (p.lse && warp == 0)
+    if (p.lse && cw == 0)
         p.lse[((size_t)b * p.Hq + head) * N + node] = l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+    TL_END(p.trace_idx, 2);
 }
 
+// Launch with programmatic stream serialisation and, when cluster > 0, thread-block clusters of that size.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    cfg.numAttrs = 1;
+    if (cluster > 0) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    cfg.attrs = attr;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
@@ -855,7 +1052,7 @@ extern "C" int vispec_debug_timeline(unsigned long long* host, int reset) {
     if (reset) {
         g_trace_launch = 0;
         static unsigned long long init[4096][4];
-        for (int i = 0; i < 4096; ++i) { init[i][0] = ~0ull; init[i][1] = 0; init[i][2] = ~0ull; init[i][3] = ~0ull; }
+        for (int i = 0; i < 4096; ++i) { init[i][0] = ~0ull; init[i][1] = 0; init[i][2] = 0; init[i][3] = ~0ull; }
         return cudaMemcpyToSymbol(g_timeline, init, sizeof(init)) == cudaSuccess ? 0 : -1;
     }
     return cudaMemcpyFromSymbol(host, g_timeline, sizeof(g_timeline)) == cudaSuccess ? 0 : -1;
@@ -863,6 +1060,36 @@ extern "C" int vispec_debug_timeline(unsigned long long* host, int reset) {
 #endif
 
 static size_t tc5_partial_bytes(int grid, int rows) { return (size_t)2 * grid * rows * (D * 4 + 8); }
+
+// Largest number of co-resident clusters of each size (index: PAIR, cluster size), found once per device.
+static int g_max_clusters[2][9];
+
+static int query_max_clusters(bool pair, int k) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(k * 64); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = SMEM_ALLOC;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = k; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    cudaError_t e = pair ? cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<true, true>, &cfg)
+                         : cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<false, true>, &cfg);
+    if (e != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
+// Cluster size for the cluster form, or 0 when the even split with partials in global memory serves better:
+// one cluster per unit, all clusters co-resident, and most of the SMs in use.
+static int tc5_cluster_size(const AttnArgs& a, int units) {
+    if (a.tc5_path == 1) return 0;
+    const bool pair = (a.Hq / a.Hkv) * a.N <= 64;
+    int best = 0;
+    for (int k = 1; k <= 8; ++k)
+        if (units * k <= a.sm_count && g_max_clusters[pair][k] >= units) best = k;
+    if (best == 0) return 0;
+    if (a.tc5_path == 2) return best;
+    return (units * best * 4 >= a.sm_count * 3) ? best : 0;
+}
 
 bool attn_tc5_supports(const AttnArgs& a) {
     if (!(a.D == 128 && a.k_map && a.v_map && a.B > 0 && a.B <= kMaxB)) return false;
@@ -876,9 +1103,19 @@ bool attn_tc5_supports(const AttnArgs& a) {
 }
 
 cudaError_t init_attn_tc5() {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
+    cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attn_tc5_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
+    e = cudaFuncSetAttribute(attn_tc5_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc5_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc5_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
+    if (e != cudaSuccess) return e;
+    for (int k = 1; k <= 8; ++k) { g_max_clusters[0][k] = query_max_clusters(false, k); g_max_clusters[1][k] = query_max_clusters(true, k); }
+    // The merge blocks must be able to join an SM that an attention CTA has configured for maximum shared memory.
+    e = cudaFuncSetAttribute(attn_tc5_merge_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_tc5_merge_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
 }
 
 cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches) {
@@ -889,7 +1126,8 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     const int n_mblocks = pair ? 1 : (rows_total + 127) / 128;
     const int units = a.B * a.Hkv * n_mblocks;
     const long long t_max = (long long)units * ((a.S_max + STEP - 1) / STEP);
-    const int grid = (int)(t_max < a.sm_count ? t_max : a.sm_count);
+    const int ck = tc5_cluster_size(a, units);
+    const int grid = ck > 0 ? units * ck : (int)(t_max < a.sm_count ? t_max : a.sm_count);
 
     Tc5Params p;
     p.q = (const __nv_bfloat16*)a.q; p.kv_len = a.kv_len; p.mask = a.mask;
@@ -906,12 +1144,21 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
 #else
     p.trace_idx = 0;
 #endif
-    cudaError_t err = pair ? launch_pdl(attn_tc5_kernel<true>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, *a.k_map, *a.v_map, p)
-                           : launch_pdl(attn_tc5_kernel<false>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, *a.k_map, *a.v_map, p);
+    cudaError_t err;
+    if (ck > 0) {
+        // cluster form: the CTAs of a unit merge their partials through distributed shared memory; one launch
+        err = pair ? launch_pdl(attn_tc5_kernel<true, true>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, ck, *a.k_map, *a.v_map, p)
+                   : launch_pdl(attn_tc5_kernel<false, true>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, ck, *a.k_map, *a.v_map, p);
+        if (err != cudaSuccess) return err;
+        ++*n_launches;
+        return cudaSuccess;
+    }
+    err = pair ? launch_pdl(attn_tc5_kernel<true, false>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, 0, *a.k_map, *a.v_map, p)
+               : launch_pdl(attn_tc5_kernel<false, false>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, 0, *a.k_map, *a.v_map, p);
     if (err != cudaSuccess) return err;
     ++*n_launches;
-    err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 2), dim3(256), 0, st, p)
-               : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 4), dim3(256), 0, st, p);
+    err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p)
+               : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 8), dim3(128), 0, st, 0, p);
     if (err != cudaSuccess) return err;
     ++*n_launches;
     return cudaSuccess;

@@ -125,6 +125,9 @@ int vispec_ctx_set_option(vispec_ctx* c, int option, int value) {
     switch (option) {
         case VISPEC_OPT_EARLY_PREFETCH: c->early_prefetch = value != 0; return VISPEC_OK;
         case VISPEC_OPT_FORCE_GENERIC: c->force_generic = value != 0; return VISPEC_OK;
+        case VISPEC_OPT_SPLIT_FORM:
+            if (value < 0 || value > 2) return VISPEC_E_RANGE;
+            c->tc5_path = value; return VISPEC_OK;
         default: return VISPEC_E_UNSUPPORTED;
     }
 }
@@ -189,6 +192,7 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
     a.scale = scale; a.ws = c->ws; a.ws_bytes = c->ws_bytes; a.status = c->d_status;
     a.sm_count = c->sm_count;
     a.early_prefetch = c->early_prefetch;
+    a.tc5_path = c->tc5_path;
     a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
     int n = 0;
     cudaError_t err = (!c->force_generic && attn_tc5_supports(a)) ? launch_attn_tc5(a, (cudaStream_t)stream, &n)

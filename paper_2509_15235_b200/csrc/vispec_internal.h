@@ -21,6 +21,7 @@ struct vispec_ctx {
     uint64_t launches = 0;
     bool force_generic = false;     // VISPEC_OPT_FORCE_GENERIC (or VISPEC_FORCE_GENERIC=1 at context creation)
     bool early_prefetch = true;     // VISPEC_OPT_EARLY_PREFETCH
+    int tc5_path = 0;               // VISPEC_OPT_SPLIT_FORM: 0 automatic, 1 partials in global memory, 2 clusters
 };
 
 namespace vispec {
@@ -54,6 +55,7 @@ struct AttnArgs {
     int* status;
     int sm_count;
     bool early_prefetch;   // committed-prefix tiles may be read before the preceding kernel has completed
+    int tc5_path;          // 0 automatic, 1 partials in global memory + merge kernel, 2 clusters where possible
     const CUtensorMap* k_map; const CUtensorMap* v_map;
 };
 // Generic split-KV kernel on warp-level tensor-core instructions (any supported shape).

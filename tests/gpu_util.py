@@ -29,12 +29,14 @@ def u64_host(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().numpy().view(np.uint64)
 
 
-def run_attn(q, k, v, kv_len, mask, scale, want_lse=True, B_max=None, N_max=None):
+def run_attn(q, k, v, kv_len, mask, scale, want_lse=True, B_max=None, N_max=None, split_form=0):
     """One attention call through the C ABI.  Inputs are numpy (bf16 bits / int32 / uint64).
     Returns (out float32 [B,N,Hq,D], lse float32 [B,Hq,N] or None, status word)."""
     B, N, Hq, D = q.shape
     _, Hkv, S_max, _ = k.shape
     ctx = binding.VerifyContext(B_max or max(B, 1), N_max or N, Hq, Hkv, D, S_max, 1)
+    if split_form:
+        ctx.ctx_set_option(binding.OPT_SPLIT_FORM, split_form)
     kd, vd = bf16_dev(k), bf16_dev(v)
     ctx.cache_register(0, kd, vd)
     qd = bf16_dev(q)

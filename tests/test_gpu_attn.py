@@ -22,8 +22,8 @@ def gu():
     return gpu_util
 
 
-def _check(gu, q, k, v, kv_len, mask, scale, rows=None):
-    out, lse, status = gu.run_attn(q, k, v, kv_len, mask, scale)
+def _check(gu, q, k, v, kv_len, mask, scale, split_form=0):
+    out, lse, status = gu.run_attn(q, k, v, kv_len, mask, scale, split_form=split_form)
     want, want_lse = oracle.tree_attn(q, k, v, kv_len, mask, scale)
     assert status == 0
     assert not np.isnan(out).any()
@@ -58,7 +58,8 @@ def test_tiny_config_full_parity(gu):
     (4, 2, 128, 31, 1000, 1088),  # the paper's 30-token tree plus root
     (3, 3, 128, 65, 130, 256),    # two mask words
 ])
-def test_shapes_span_tiles_tails_and_group_sizes(gu, Hq, Hkv, D, N, S, S_max):
+@pytest.mark.parametrize("split_form", [0, 1, 2])
+def test_shapes_span_tiles_tails_and_group_sizes(gu, Hq, Hkv, D, N, S, S_max, split_form):
     rng = np.random.Generator(np.random.Philox(Hq * 1000 + N))
     B = 2
     q = synth.normal_bf16((B, N, Hq, D), 1 + N)
@@ -67,7 +68,7 @@ def test_shapes_span_tiles_tails_and_group_sizes(gu, Hq, Hkv, D, N, S, S_max):
     kv_len = np.array([S, max(0, S - 61)], dtype=np.int32)
     parents = np.stack([synth.draw_tree(N, 6, 4, rng) for _ in range(B)])
     mask, _, _ = oracle.tree_mask(parents)
-    _check(gu, q, k, v, kv_len, mask, 1 / math.sqrt(D))
+    _check(gu, q, k, v, kv_len, mask, 1 / math.sqrt(D), split_form=split_form)
 
 
 def test_arbitrary_mask_bits_all_ones_and_zero_rows(gu):
@@ -172,11 +173,13 @@ def test_host_side_argument_errors(gu):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("split_form", [1, 2])
 @pytest.mark.parametrize("name", ["llava7b", "qwen7b"])
-def test_full_size_layer_parity(gu, name):
-    """One whole layer at benchmark size, every output element against the oracle."""
+def test_full_size_layer_parity(gu, name, split_form):
+    """One whole layer at benchmark size, every output element against the oracle, for both ways of
+    combining the pieces of a head (partials + merge kernel; clusters)."""
     cfg = synth.get_config(name)
-    _check(gu, *_case(cfg, layer=1), 1 / math.sqrt(cfg.D))
+    _check(gu, *_case(cfg, layer=1), 1 / math.sqrt(cfg.D), split_form=split_form)
 
 
 def test_full_size_batched_variable_length_parity(gu):
