@@ -13,10 +13,12 @@
 // the partials of each unit.  Both kernels derive the same schedule from kv_len on the device, so the
 // host never reads lengths.
 //
-// Inside a CTA the 6 warps are specialised:
+// Inside a CTA the 7 warps are specialised:
 //   warp 0     TMA producer: K ring and V ring of 128-token stages (32 KB each, 128-byte swizzle); it runs
 //              ahead across segment boundaries
-//   warp 1     tensor-core issuer (one thread): S = Q K^T and O += P V as 128x128x16 tcgen05.mma, owns TMEM
+//   warp 1     issuer (one thread) of S = Q K^T as 128x128x16 tcgen05.mma; owns the TMEM allocation
+//   warp 6     issuer (one thread) of O += P V; the two chains wait on different barriers, so each has its own
+//              thread and neither's waits delay the other's instructions
 //   warps 2-5  softmax: thread <-> TMEM lane, i.e. one thread per accumulator row, no shuffles; they also
 //              load Q at the start of every segment and run the segment epilogue
 // TMEM map (512 columns x 128 lanes): S[0] 0..127, S[1] 128..255, O 256..383, P[0] 384..447, P[1] 448..511.
@@ -53,7 +55,7 @@ constexpr int STEP = 128;                      // tokens per pipeline step = row
 constexpr int HALF_BYTES = STEP * 128;         // one d-half (64 columns) of a stage: 128 rows x 128 B
 constexpr int STAGE_BYTES = 2 * HALF_BYTES;    // 32 KB
 constexpr int NSK = 3, NSV = 3;
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr int kMaxB = 64;                      // sequences per call this kernel takes
 constexpr int SMEM_K = 0;
 constexpr int SMEM_V = SMEM_K + NSK * STAGE_BYTES;
@@ -490,38 +492,15 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ================= tensor-core issuer =================
+        // ================= issuer of the S products =================
         if (lane == 0 && active) {
             constexpr uint32_t IDESC_S = instr_desc(0);            // B = K stage, K-major
-            constexpr uint32_t IDESC_O = instr_desc(1);            // B = V stage, MN-major
             constexpr uint32_t DESC_HI = desc_hi(1024);            // 8 rows x 128 B between row groups, everywhere
-            auto issue_pv = [&](int u, uint32_t acc) -> bool {
-                const int bu = u & 1, sv = u % NSV;
-                TRACE(1, u, 3);
-                if (!mbar_wait(bar(B_PFULL + bu), (u >> 1) & 1, abort_flag)) return false;
-                TRACE(1, u, 4);
-                if (!mbar_wait(bar(B_VFULL + sv), (u / NSV) & 1, abort_flag)) return false;
-                TRACE(1, u, 5);
-                tc_fence_after();
-                const uint32_t vb = desc_lo(base + SMEM_V + sv * STAGE_BYTES, HALF_BYTES);
-#pragma unroll
-                for (int ks = 0; ks < STEP / 16; ++ks)      // 16 tokens per instruction: 8 P columns, 16 V rows (2 KB)
-                    tc_mma_ts(tmem + COL_O, tmem + COL_P + bu * 64 + ks * 8, vb + ks * 128, DESC_HI, IDESC_O,
-                              (acc || ks > 0) ? 1u : 0u);
-                tc_commit(bar(B_VEMPTY + sv));
-                tc_commit(bar(B_PVDONE + bu));
-                TRACE(1, u, 6);
-                return true;
-            };
-            bool ok = true, have_prev = false;
-            uint32_t acc_prev = 0;
+            bool ok = true;
             int it = 0, seg = 0;
             SegIter si = make_iter();
             Seg sg;
             while (ok && si.next(sg)) {
-                // Q of this segment is loaded only after the previous segment's epilogue, which waits for that
-                // segment's last PV product: issue it before waiting for Q
-                if (have_prev) { ok = issue_pv(it - 1, acc_prev); have_prev = false; if (!ok) break; }
                 if (!mbar_wait(bar(B_QFULL), seg & 1, abort_flag)) { ok = false; break; }
                 for (int t = 0; t < sg.n && ok; ++t, ++it) {
                     const int bs = it & 1, sk = it % NSK;
@@ -541,13 +520,39 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     tc_commit(bar(B_KEMPTY + sk));
                     tc_commit(bar(B_SFULL + bs));
                     TRACE(1, it, 2);
-                    if (have_prev) ok = issue_pv(it - 1, acc_prev);
-                    have_prev = true;
-                    acc_prev = t > 0 ? 1u : 0u;                 // the first product of a segment starts a fresh O
                 }
                 ++seg;
             }
-            if (ok && have_prev) issue_pv(it - 1, acc_prev);
+        }
+        __syncwarp();
+    } else if (warp == 6) {
+        // ================= issuer of the PV products =================
+        if (lane == 0 && active) {
+            constexpr uint32_t IDESC_O = instr_desc(1);            // B = V stage, MN-major
+            constexpr uint32_t DESC_HI = desc_hi(1024);
+            bool ok = true;
+            int u = 0;
+            SegIter si = make_iter();
+            Seg sg;
+            while (ok && si.next(sg)) {
+                for (int t = 0; t < sg.n; ++t, ++u) {
+                    const int bu = u & 1, sv = u % NSV;
+                    TRACE(1, u, 3);
+                    if (!mbar_wait(bar(B_PFULL + bu), (u >> 1) & 1, abort_flag)) { ok = false; break; }
+                    TRACE(1, u, 4);
+                    if (!mbar_wait(bar(B_VFULL + sv), (u / NSV) & 1, abort_flag)) { ok = false; break; }
+                    TRACE(1, u, 5);
+                    tc_fence_after();
+                    const uint32_t vb = desc_lo(base + SMEM_V + sv * STAGE_BYTES, HALF_BYTES);
+#pragma unroll
+                    for (int ks = 0; ks < STEP / 16; ++ks)      // 16 tokens per instruction: 8 P columns, 16 V rows (2 KB)
+                        tc_mma_ts(tmem + COL_O, tmem + COL_P + bu * 64 + ks * 8, vb + ks * 128, DESC_HI, IDESC_O,
+                                  (t > 0 || ks > 0) ? 1u : 0u);   // the first product of a segment starts a fresh O
+                    tc_commit(bar(B_VEMPTY + sv));
+                    tc_commit(bar(B_PVDONE + bu));
+                    TRACE(1, u, 6);
+                }
+            }
         }
         __syncwarp();
     } else {
