@@ -13,14 +13,16 @@
 // the partials of each unit.  Both kernels derive the same schedule from kv_len on the device, so the
 // host never reads lengths.
 //
-// Inside a CTA the 7 warps are specialised:
+// Inside a CTA the 12 warps are specialised:
 //   warp 0     TMA producer: K ring and V ring of 128-token stages (32 KB each, 128-byte swizzle); it runs
 //              ahead across segment boundaries
 //   warp 1     issuer (one thread) of S = Q K^T as 128x128x16 tcgen05.mma; owns the TMEM allocation
-//   warp 6     issuer (one thread) of O += P V; the two chains wait on different barriers, so each has its own
+//   warp 2     issuer (one thread) of O += P V; the two chains wait on different barriers, so each has its own
 //              thread and neither's waits delay the other's instructions
-//   warps 2-5  softmax: thread <-> TMEM lane, i.e. one thread per accumulator row, no shuffles; they also
-//              load Q at the start of every segment and run the segment epilogue
+//   warp 3     derives the schedule from kv_len, then idles
+//   warps 4-11 softmax: thread <-> TMEM lane; warps w and w+4 share the same 32 accumulator rows and each takes
+//              half of a step's columns (the row maximum is exchanged through shared memory), so a row costs
+//              no shuffles; they also load Q at the start of every segment and run the segment epilogue
 // TMEM map (512 columns x 128 lanes): S[0] 0..127, S[1] 128..255, O 256..383, P[0] 384..447, P[1] 448..511.
 // P (bf16, packed two per column) is the A operand of the PV product and never touches shared memory; Q
 // sits in shared memory in the same swizzled K-major layout as a K stage.  S and P are double-buffered: S
@@ -55,14 +57,15 @@ constexpr int STEP = 128;                      // tokens per pipeline step = row
 constexpr int HALF_BYTES = STEP * 128;         // one d-half (64 columns) of a stage: 128 rows x 128 B
 constexpr int STAGE_BYTES = 2 * HALF_BYTES;    // 32 KB
 constexpr int NSK = 3, NSV = 3;
-constexpr int kThreads = 224;
-constexpr int kMaxB = 64;                      // sequences per call this kernel takes
+constexpr int kThreads = 384;                  // 12 warps: producer, two issuers, one spare, eight softmax
+constexpr int kSmx = 256;                      // softmax threads
+constexpr int kMaxB = 32;                      // sequences per call this kernel takes
 constexpr int SMEM_K = 0;
 constexpr int SMEM_V = SMEM_K + NSK * STAGE_BYTES;
 constexpr int SMEM_Q = SMEM_V + NSV * STAGE_BYTES;             // Q tile, 128 rows, laid out like a K stage; between
                                                                // segments it is the PAIR exchange [32 col4][64 rows] float4
-constexpr int SMEM_XST = SMEM_Q + STAGE_BYTES;                 // PAIR exchange of statistics: 64 float2
-constexpr int SMEM_BAR = SMEM_XST + 64 * 8;
+constexpr int SMEM_XM = SMEM_Q + STAGE_BYTES;                  // 512 floats: tile maxima / row statistics exchanged between threads
+constexpr int SMEM_BAR = SMEM_XM + 2048;
 constexpr int BAR_BYTES = 256;
 constexpr int SMEM_SCHED = SMEM_BAR + BAR_BYTES;
 constexpr uint32_t TMEM_COLS = 512;
@@ -72,7 +75,7 @@ constexpr long long kWaitCycles = 1500000000LL;                // ~0.8 s at 1.9 
 
 enum { B_KFULL = 0, B_KEMPTY = B_KFULL + NSK, B_VFULL = B_KEMPTY + NSK, B_VEMPTY = B_VFULL + NSV,
        B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2,
-       B_QFULL = B_PVDONE + 2, B_XCH = B_QFULL + 1, B_XFREE = B_XCH + 1,
+       B_QFULL = B_PVDONE + 2, B_PAIRX = B_QFULL + 1, B_XCH = B_PAIRX + 4, B_XFREE = B_XCH + 1,
        B_EPI = B_XFREE + 1, B_CL1 = B_EPI + 1, B_COUNT = B_CL1 + 1 };
 static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block too small");
 
@@ -84,7 +87,7 @@ struct Sched {
     int units;             // units with at least one step
 };
 constexpr int SMEM_TOTAL = SMEM_SCHED + (int)sizeof(Sched);
-constexpr int SMEM_ALLOC = SMEM_TOTAL + 1024;                  // slack to align the base to 1024 B
+constexpr int SMEM_ALLOC = SMEM_TOTAL;                         // the base must come out 1024-byte aligned (checked)
 static_assert(SMEM_ALLOC <= 232448, "over the 227 KB a CTA may have");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -222,6 +225,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr),
+          "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -261,7 +273,7 @@ __device__ long long g_trace[3][64][8];
 __device__ long long g_trace_misc[16];
 __device__ int g_trace_cta = 0;
 #define TRACE(role, step, slot) do { if (blockIdx.x == g_trace_cta && (step) < 64) g_trace[role][step][slot] = clock64(); } while (0)
-#define TRACE_MISC(slot) do { if (blockIdx.x == g_trace_cta && threadIdx.x == 64) g_trace_misc[slot] = clock64(); } while (0)
+#define TRACE_MISC(slot) do { if (blockIdx.x == g_trace_cta && threadIdx.x == 128) g_trace_misc[slot] = clock64(); } while (0)
 // Per-launch timeline in globaltimer nanoseconds: [launch][0/1] attention first start / last end, [2/3] merge.
 __device__ unsigned long long g_timeline[4096][4];
 __device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
@@ -382,14 +394,17 @@ template <bool PAIR, bool CL>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const Tc5Params p) {
     constexpr int ROWS = PAIR ? 64 : 128;      // distinct query rows per CTA
-    constexpr int NCOL = PAIR ? 64 : 128;      // tokens of a step one thread handles
-    extern __shared__ unsigned char smem_raw[];
+    constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
+    extern __shared__ __align__(1024) unsigned char sm[];
     TRACE_MISC(0);
     TL_START(p.trace_idx, 0);
     CTA_T(0);
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    unsigned char* sm = smem_raw + (base - raw);
+    const uint32_t base = smem_u32(sm);
+    if (base & 1023u) {
+        // the swizzled tiles need a 1024-byte aligned base; every CTA sees the same base, so all of them leave
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)VISPEC_E_UNSUPPORTED);
+        return;
+    }
     const uint32_t bars = base + SMEM_BAR;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + SMEM_BAR + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SMEM_BAR + B_COUNT * 8 + 8);
@@ -405,12 +420,13 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         for (int i = 0; i < NSK; ++i) { mbar_init(bar(B_KFULL + i), 1); mbar_init(bar(B_KEMPTY + i), 1); }
         for (int i = 0; i < NSV; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(B_SFULL + i), 1); mbar_init(bar(B_SFREE + i), 128);
-            mbar_init(bar(B_PFULL + i), 128); mbar_init(bar(B_PVDONE + i), 1);
+            mbar_init(bar(B_SFULL + i), 1); mbar_init(bar(B_SFREE + i), kSmx);
+            mbar_init(bar(B_PFULL + i), kSmx); mbar_init(bar(B_PVDONE + i), 1);
         }
-        mbar_init(bar(B_QFULL), 128);
-        mbar_init(bar(B_XCH), 64); mbar_init(bar(B_XFREE), 64);
-        mbar_init(bar(B_EPI), 128);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(B_PAIRX + i), 64);
+        mbar_init(bar(B_QFULL), kSmx);
+        mbar_init(bar(B_XCH), 128); mbar_init(bar(B_XFREE), 128);
+        mbar_init(bar(B_EPI), kSmx);
         mbar_init(bar(B_CL1), CL ? cluster_size() : 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -419,7 +435,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (warp == 2) sched_build(sched, p, lane);
+    if (warp == 3) sched_build(sched, p, lane);
     pdl_launch_dependents();
     if (!p.early) pdl_wait();
     TRACE_MISC(1);
@@ -525,7 +541,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             }
         }
         __syncwarp();
-    } else if (warp == 6) {
+    } else if (warp == 2) {
         // ================= issuer of the PV products =================
         if (lane == 0 && active) {
             constexpr uint32_t IDESC_O = instr_desc(1);            // B = V stage, MN-major
@@ -555,14 +571,18 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             }
         }
         __syncwarp();
-    } else {
-        // ================= softmax: one thread per accumulator row =================
-        const int sp = warp & 3;
-        const int tl = sp * 32 + lane;                       // TMEM lane
-        const int half = PAIR ? (tl >> 6) : 0;               // PAIR: which 64 tokens of each step
-        const int lrow = PAIR ? (tl & 63) : tl;              // row within the block
+    } else if (warp >= 4) {
+        // ================= softmax: two threads per accumulator row, each takes half of a step's columns =================
+        const int sp = warp & 3;                              // TMEM lane quarter of this warp
+        const int ch = (warp - 4) >> 2;                       // which half of the row's columns (and of the O columns)
+        const int tl = sp * 32 + lane;                        // TMEM lane
+        const int half = PAIR ? (tl >> 6) : 0;                // PAIR: which 64 tokens of each step the lane's row copy covers
+        const int lrow = PAIR ? (tl & 63) : tl;               // row within the block
         const uint32_t lane_addr = tmem + ((uint32_t)(32 * sp) << 16);
-        const int st = tid - 64;                              // 0..127
+        const int st = tid - 128;                             // 0..255
+        float* xm = reinterpret_cast<float*>(sm + SMEM_XM);   // [2 step parities][2 column halves][128 lanes] tile maxima;
+                                                              // in the epilogue: [0..255] l by (ch, lane), [256..383] m by lane
+        int px = 0;                                           // phases of the pair barrier used so far
         pdl_wait();                                           // q, tree_mask and every output come after the preceding kernel
 
         // rejected sequences (kv_len < 0 or kv_len + N > S_max): zero output, -inf lse, status word
@@ -574,42 +594,49 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 any_bad = true;
                 const int vecs = N * p.Hq * (D / 8);
                 uint4* o = reinterpret_cast<uint4*>(p.out + (size_t)b * N * p.Hq * D);
-                for (int i = cta * 128 + st; i < vecs; i += (int)gridDim.x * 128) o[i] = make_uint4(0, 0, 0, 0);
+                for (int i = cta * kSmx + st; i < vecs; i += (int)gridDim.x * kSmx) o[i] = make_uint4(0, 0, 0, 0);
                 if (p.lse)
-                    for (int i = cta * 128 + st; i < N * p.Hq; i += (int)gridDim.x * 128) p.lse[(size_t)b * p.Hq * N + i] = -INFINITY;
+                    for (int i = cta * kSmx + st; i < N * p.Hq; i += (int)gridDim.x * kSmx) p.lse[(size_t)b * p.Hq * N + i] = -INFINITY;
             }
             if (any_bad && cta == 0 && st == 0) atomicCAS(p.status, 0, (int)VISPEC_E_RANGE);
         }
 
         // Q of a segment -> shared memory, rows in the swizzled K-major layout of a K stage (PAIR: rows 64-127
-        // repeat rows 0-63).  Thread t moves 16-byte chunk t%16 of rows t/16, t/16 + 8, ...
+        // repeat rows 0-63).  Thread t moves 16-byte chunk t%16 of rows t/16, t/16 + 16, ...
         auto load_q = [&](const Seg& sg, int seg) -> bool {
             if (PAIR && seg > 0) {
                 // the tile doubles as the exchange area of the previous segment's epilogue
                 if (!mbar_wait_warp(bar(B_XFREE), (seg - 1) & 1, abort_flag)) return false;
             }
-            constexpr int ITEMS = ROWS * 16 / 128;
-            const int ch = st & 15;
+            constexpr int ITEMS = ROWS * 16 / kSmx;
+            const int qc = st & 15;
             uint4 v[ITEMS];
 #pragma unroll
             for (int k = 0; k < ITEMS; ++k) {
-                const int row = sg.mblock * 128 + (st >> 4) + 8 * k;
+                const int row = sg.mblock * 128 + (st >> 4) + 16 * k;
                 v[k] = make_uint4(0, 0, 0, 0);
                 if (row < rows_total) {
                     const int node = row / G, head = sg.kvh * G + row % G;
-                    v[k] = *(reinterpret_cast<const uint4*>(p.q + (((size_t)sg.b * N + node) * p.Hq + head) * D) + ch);
+                    v[k] = *(reinterpret_cast<const uint4*>(p.q + (((size_t)sg.b * N + node) * p.Hq + head) * D) + qc);
                 }
             }
 #pragma unroll
             for (int k = 0; k < ITEMS; ++k) {
-                const int r = (st >> 4) + 8 * k;
-                unsigned char* dst = sm + SMEM_Q + (ch >> 3) * HALF_BYTES + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
+                const int r = (st >> 4) + 16 * k;
+                unsigned char* dst = sm + SMEM_Q + (qc >> 3) * HALF_BYTES + r * 128 + (((qc & 7) ^ (r & 7)) << 4);
                 *reinterpret_cast<uint4*>(dst) = v[k];
                 if (PAIR) *reinterpret_cast<uint4*>(dst + 64 * 128) = v[k];
             }
             fence_async_smem();
             mbar_arrive(bar(B_QFULL));
             return true;
+        };
+        // Meeting of the two warps that share this warp's rows (bounded; warp-uniform result).
+        auto pair_sync = [&]() -> bool {
+            mbar_arrive(bar(B_PAIRX + sp));
+            const bool r = mbar_wait_warp(bar(B_PAIRX + sp), px & 1, abort_flag);
+            ++px;
+            return r;
         };
 
         if (active) {
@@ -618,7 +645,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             int it = 0, seg = 0;
             bool ok = true;
             float4* xch = reinterpret_cast<float4*>(sm + SMEM_Q);
-            float2* xst = reinterpret_cast<float2*>(sm + SMEM_XST);
             while (ok && si.next(sg)) {
                 // every S product of the previous segment has been consumed by now, so Q may be replaced
                 if (!load_q(sg, seg)) { ok = false; break; }
@@ -637,111 +663,117 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     if (N < 64) mk0 &= (1ull << N) - 1;
                     if (N < 128) mk1 &= N > 64 ? (1ull << (N - 64)) - 1 : 0ull;
                 }
+                // m_ref and has_o are the same in both threads of a row; l_run covers this thread's columns only
                 float m_ref = -INFINITY, l_run = 0.f;
                 bool has_o = false;
 
                 for (int t = 0; t < sg.n; ++t, ++it) {
                     const int bs = it & 1;
                     const int tok0 = (sg.st0 + t) * STEP;
-                    if (tid == 64) TRACE(2, it, 0);
+                    if (tid == 128) TRACE(2, it, 0);
                     if (!mbar_wait_warp(bar(B_SFULL + bs), (it >> 1) & 1, abort_flag)) { ok = false; break; }
-                    if (tid == 64) TRACE(2, it, 1);
+                    if (tid == 128) TRACE(2, it, 1);
                     tc_fence_after();
-                    uint32_t sraw[NCOL];
+                    uint32_t sraw[NC];
 #pragma unroll
-                    for (int ch = 0; ch < NCOL / 32; ++ch) tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + ch * 32, sraw + ch * 32);
+                    for (int c = 0; c < NC / 32; ++c) tmem_ld32(lane_addr + COL_S + bs * 128 + half * 64 + ch * NC + c * 32, sraw + c * 32);
                     tmem_wait_ld();
                     tc_fence_before();
                     mbar_arrive(bar(B_SFREE + bs));             // the S product of step it+2 may overwrite the buffer
-                    if (tid == 64) TRACE(2, it, 2);
+                    if (tid == 128) TRACE(2, it, 2);
 
-                    const int j0 = tok0 + half * 64;                        // first token this thread looks at
-                    const bool valid = j0 < total;
-                    float tmax = -INFINITY;
+                    const int jr = tok0 + half * 64;                        // first token of the row's part of the tile
+                    const int j0 = jr + ch * NC;                            // first token this thread looks at
+                    const bool row_valid = jr < total, valid = j0 < total;
+                    float lmax = -INFINITY;
                     if (valid) {
-                        if (j0 + NCOL > S) {
+                        if (j0 + NC > S) {
                             // reaches past the committed prefix: ancestor bits for tree rows, nothing beyond them
-                            // bit c of (a0, a1): column c may be attended to (prefix column, or visible tree node)
+                            // bit c of a0: column c may be attended to (prefix column, or visible tree node)
                             const int t0 = j0 - S;                           // tree index of column 0 (may be negative)
                             uint64_t a0, a1;
                             if (t0 >= 0) shr128(mk0, mk1, t0, a0, a1); else shl128_fill(mk0, mk1, -t0, a0, a1);
 #pragma unroll
-                            for (int c = 0; c < NCOL; ++c)
-                                if (!(((c < 64 ? a0 : a1) >> (c & 63)) & 1ull)) sraw[c] = 0xff800000u;   // -inf
+                            for (int c = 0; c < NC; ++c)
+                                if (!((a0 >> c) & 1ull)) sraw[c] = 0xff800000u;   // -inf
                         }
                         float mx[8];
 #pragma unroll
                         for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sraw[c]);
 #pragma unroll
-                        for (int c = 8; c < NCOL; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sraw[c]));
+                        for (int c = 8; c < NC; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sraw[c]));
                         // the scale is positive, so it commutes with the maximum
-                        tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
+                        lmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
                     }
+                    // the row's maximum over the tile: the other thread of the row has the other columns
+                    xm[(it & 1) * 256 + ch * 128 + tl] = lmax;
+                    if (!pair_sync()) { ok = false; break; }
+                    const float tmax = fmaxf(lmax, xm[(it & 1) * 256 + (ch ^ 1) * 128 + tl]);
                     // move the reference maximum only when the tile exceeds it by more than the gap
                     float alpha = 1.f;
                     bool rescale = false;
-                    if (valid && tmax > m_ref + kRescaleGap) {          // also true on the first finite tile (m_ref = -inf)
+                    if (row_valid && tmax > m_ref + kRescaleGap) {      // also true on the first finite tile (m_ref = -inf)
                         alpha = exp2f(m_ref - tmax);                     // 0 when m_ref = -inf
                         m_ref = tmax;
                         l_run *= alpha;
                         rescale = has_o;
                     }
                     if (__any_sync(0xffffffffu, rescale)) {
-                        // O was last written by the PV product of step it-1 (same segment: has_o is set)
+                        // O was last written by the PV product of step it-1 (same segment: has_o is set); this thread
+                        // rescales its half of the row's columns
                         if (!mbar_wait_warp(bar(B_PVDONE + (bs ^ 1)), ((it - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
+                        for (int c = 0; c < 2; ++c) {
                             uint32_t o[32];
-                            tmem_ld32(lane_addr + COL_O + ch * 32, o);
+                            tmem_ld32(lane_addr + COL_O + ch * 64 + c * 32, o);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                            tmem_st32(lane_addr + COL_O + ch * 32, o);
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st32(lane_addr + COL_O + ch * 64 + c * 32, o);
                         }
                     }
-                    if (tid == 64) TRACE(2, it, 3);
-                    // P = exp2(scale * s - m_ref) as bf16 pairs into the P columns (column c holds tokens 2c, 2c+1)
-                    uint32_t pd[NCOL / 2];
+                    if (tid == 128) TRACE(2, it, 3);
+                    // P = exp2(scale * s - m_ref) as bf16 pairs (column c of P holds tokens 2c, 2c+1)
+                    uint32_t pd[NC / 2];
                     if (valid) {
                         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
                         float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                        for (int c = 0; c < NCOL / 2; ++c) {
+                        for (int c = 0; c < NC / 2; ++c) {
                             const float e0 = exp2f(fmaf(__uint_as_float(sraw[2 * c]), p.scale_log2, -m_use));
                             const float e1 = exp2f(fmaf(__uint_as_float(sraw[2 * c + 1]), p.scale_log2, -m_use));
                             sum0 += e0; sum1 += e1;
                             pd[c] = pack_bf16(e0, e1);
                         }
                         l_run += sum0 + sum1;
-                        has_o = true;
                     } else {
 #pragma unroll
-                        for (int c = 0; c < NCOL / 2; ++c) pd[c] = 0u;
+                        for (int c = 0; c < NC / 2; ++c) pd[c] = 0u;
                     }
+                    if (row_valid) has_o = true;
                     // P[bs] is free once the PV product of step it-2 has completed
                     if (it >= 2) {
                         if (!mbar_wait_warp(bar(B_PVDONE + bs), ((it >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                     }
                     if (PAIR) {
-                        // block-diagonal P: this row weighs only its own half's tokens, the other 32 columns are zero
-                        uint32_t zero[32];
+                        // block-diagonal P: the row weighs only its own half's tokens, the other 32 columns are zero
+                        uint32_t zero[16];
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) zero[c] = 0u;
-                        tmem_st32(lane_addr + COL_P + bs * 64 + half * 32, pd);
-                        tmem_st32(lane_addr + COL_P + bs * 64 + (half ^ 1) * 32, zero);
+                        for (int c = 0; c < 16; ++c) zero[c] = 0u;
+                        tmem_st16(lane_addr + COL_P + bs * 64 + half * 32 + ch * 16, pd);
+                        tmem_st16(lane_addr + COL_P + bs * 64 + (half ^ 1) * 32 + ch * 16, zero);
                     } else {
-                        tmem_st32(lane_addr + COL_P + bs * 64, pd);
-                        tmem_st32(lane_addr + COL_P + bs * 64 + 32, pd + (NCOL / 2 - 32));
+                        tmem_st32(lane_addr + COL_P + bs * 64 + ch * 32, pd);
                     }
                     bool fail = false;
                     if (tok0 + STEP > total) {
                         // last step of the sequence: V rows past the last key may hold anything, and they meet
-                        // weight-0 columns of P in the product: clear them (thread r clears row r of the stage)
+                        // weight-0 columns of P in the product: clear them (thread r of the first 128 clears row r)
                         const int sv = it % NSV;
                         fail = !mbar_wait(bar(B_VFULL + sv), (it / NSV) & 1, abort_flag);
-                        if (!fail && tok0 + tl >= total) {
+                        if (!fail && ch == 0 && tok0 + tl >= total) {
                             unsigned char* vrow = sm + SMEM_V + sv * STAGE_BYTES + tl * 128;
 #pragma unroll
                             for (int c = 0; c < 8; ++c) {
@@ -753,46 +785,52 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     }
                     tmem_wait_st();
                     if (__any_sync(0xffffffffu, fail)) { ok = false; break; }
-                    if (tid == 64) TRACE(2, it, 5);
+                    if (tid == 128) TRACE(2, it, 5);
                     tc_fence_before();
                     mbar_arrive(bar(B_PFULL + bs));
-                    if (tid == 64) TRACE(2, it, 6);
+                    if (tid == 128) TRACE(2, it, 6);
                 }
                 if (!ok) break;
 
-                // ---- segment epilogue: wait for the last product, (PAIR) merge the two halves, write out ----
+                // ---- segment epilogue: wait for the last product, add up the row statistics, (PAIR) merge the two
+                // halves, write out.  A thread owns columns [64 ch, 64 ch + 64) of its lane's accumulator row. ----
                 TRACE_MISC(5);
                 if (sg.n > 0) ok = mbar_wait_warp(bar(B_PVDONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 TRACE_MISC(6);
-                float w_me = has_o ? 1.f : 0.f, w_other = 0.f, m_all = has_o ? m_ref : -INFINITY, l_all = l_run;
+                // (the tile-maximum slots are idle: the other thread of the row read its last one before it arrived
+                // for the last PV product)
+                xm[ch * 128 + tl] = l_run;
+                if (ch == 0) xm[256 + tl] = has_o ? m_ref : -INFINITY;
+                if (!pair_sync()) { ok = false; break; }
+                const float l_lane = xm[tl] + xm[128 + tl];                  // l of this lane's row copy
+                float w_me = has_o ? 1.f : 0.f, w_other = 0.f, m_all = has_o ? m_ref : -INFINITY, l_all = l_lane;
                 if (PAIR) {
                     if (half == 1) {
-                        // hand the raw accumulator and the statistics to the lane that owns the row (the Q tile
-                        // is idle: every S product of the segment has completed)
-                        xst[lrow] = make_float2(m_all, l_run);
+                        // hand the raw accumulator to the lane that owns the row (the Q tile is idle: every S product
+                        // of the segment has completed); the statistics are in place already
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
+                        for (int c = 0; c < 2; ++c) {
                             uint32_t o[32];
-                            tmem_ld32(lane_addr + COL_O + ch * 32, o);
+                            tmem_ld32(lane_addr + COL_O + ch * 64 + c * 32, o);
                             tmem_wait_ld();
 #pragma unroll
                             for (int c4 = 0; c4 < 8; ++c4)
-                                xch[(ch * 8 + c4) * 64 + lrow] = make_float4(__uint_as_float(o[4 * c4]), __uint_as_float(o[4 * c4 + 1]),
-                                                                            __uint_as_float(o[4 * c4 + 2]), __uint_as_float(o[4 * c4 + 3]));
+                                xch[(ch * 16 + c * 8 + c4) * 64 + lrow] = make_float4(__uint_as_float(o[4 * c4]), __uint_as_float(o[4 * c4 + 1]),
+                                                                                     __uint_as_float(o[4 * c4 + 2]), __uint_as_float(o[4 * c4 + 3]));
                         }
                         tc_fence_before();
                         mbar_arrive(bar(B_XCH));
                     } else {
                         ok = mbar_wait_warp(bar(B_XCH), seg & 1, abort_flag);
                         if (!ok) break;
-                        const float2 other = xst[lrow];
-                        m_all = fmaxf(m_all, other.x);
+                        const float m_o = xm[256 + 64 + tl], l_o = xm[64 + tl] + xm[128 + 64 + tl];
+                        m_all = fmaxf(m_all, m_o);
                         const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
                         w_me = has_o ? exp2f(m_ref - m_fin) : 0.f;
-                        w_other = exp2f(other.x - m_fin);               // 0 when the other half saw nothing
-                        l_all = l_run * w_me + other.y * w_other;
+                        w_other = exp2f(m_o - m_fin);                   // 0 when the other half saw nothing
+                        l_all = l_lane * w_me + l_o * w_other;
                     }
                 }
                 // O is only defined once a product has run (an empty cluster part never ran one): select, never
@@ -802,21 +840,21 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 if (half == 0) {
                     const bool final_out = !CL && sg.slot < 0;
                     const float inv = final_out ? (l_all > 0.f ? 1.f / l_all : 0.f) : 1.f;
-                    __nv_bfloat16* orow = p.out + (((size_t)sg.b * N + node) * p.Hq + head) * D;
-                    float4* prow = CL ? pbuf + lrow : p.part_o + (size_t)(final_out ? 0 : sg.slot) * 32 * ROWS + lrow;
+                    __nv_bfloat16* orow = p.out + (((size_t)sg.b * N + node) * p.Hq + head) * D + ch * 64;
+                    float4* prow = (CL ? pbuf : p.part_o + (size_t)(final_out ? 0 : sg.slot) * 32 * ROWS) + (size_t)ch * 16 * ROWS + lrow;
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
+                    for (int c = 0; c < 2; ++c) {
                         uint32_t o[32];
-                        tmem_ld32(lane_addr + COL_O + ch * 32, o);
+                        tmem_ld32(lane_addr + COL_O + ch * 64 + c * 32, o);
                         tmem_wait_ld();
                         float v[32];
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) v[c] = has_o ? __uint_as_float(o[c]) * w_me : 0.f;
+                        for (int e = 0; e < 32; ++e) v[e] = has_o ? __uint_as_float(o[e]) * w_me : 0.f;
                         if (PAIR) {
                             if (w_other > 0.f) {
 #pragma unroll
                                 for (int c4 = 0; c4 < 8; ++c4) {
-                                    const float4 w = xch[(ch * 8 + c4) * 64 + lrow];
+                                    const float4 w = xch[(ch * 16 + c * 8 + c4) * 64 + lrow];
                                     v[4 * c4] += w.x * w_other; v[4 * c4 + 1] += w.y * w_other;
                                     v[4 * c4 + 2] += w.z * w_other; v[4 * c4 + 3] += w.w * w_other;
                                 }
@@ -826,25 +864,27 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                             if (row_ok) {
 #pragma unroll
                                 for (int c8 = 0; c8 < 4; ++c8)
-                                    *reinterpret_cast<uint4*>(orow + ch * 32 + c8 * 8) =
+                                    *reinterpret_cast<uint4*>(orow + c * 32 + c8 * 8) =
                                         make_uint4(pack_bf16(v[8 * c8] * inv, v[8 * c8 + 1] * inv), pack_bf16(v[8 * c8 + 2] * inv, v[8 * c8 + 3] * inv),
                                                    pack_bf16(v[8 * c8 + 4] * inv, v[8 * c8 + 5] * inv), pack_bf16(v[8 * c8 + 6] * inv, v[8 * c8 + 7] * inv));
                             }
                         } else if (CL || row_ok) {
 #pragma unroll
                             for (int c4 = 0; c4 < 8; ++c4)
-                                prow[(size_t)(ch * 8 + c4) * ROWS] = make_float4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
+                                prow[(size_t)(c * 8 + c4) * ROWS] = make_float4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
                         }
                     }
-                    const float2 stat = make_float2(l_all > 0.f ? m_all : -INFINITY, l_all);
-                    if (CL) {
-                        pst[lrow] = stat;
-                    } else if (row_ok) {
-                        if (final_out) {
-                            if (p.lse) p.lse[((size_t)sg.b * p.Hq + head) * N + node] =
-                                l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
-                        } else {
-                            p.part_ml[(size_t)sg.slot * ROWS + lrow] = stat;
+                    if (ch == 0) {
+                        const float2 stat = make_float2(l_all > 0.f ? m_all : -INFINITY, l_all);
+                        if (CL) {
+                            pst[lrow] = stat;
+                        } else if (row_ok) {
+                            if (final_out) {
+                                if (p.lse) p.lse[((size_t)sg.b * p.Hq + head) * N + node] =
+                                    l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+                            } else {
+                                p.part_ml[(size_t)sg.slot * ROWS + lrow] = stat;
+                            }
                         }
                     }
                     if (PAIR) mbar_arrive(bar(B_XFREE));
@@ -867,7 +907,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                         const int row0 = cr * rp;
                         const int nrows = min(rp, ROWS - row0);
                         const uint32_t pbuf_a = base + SMEM_K, pst_a = base + SMEM_K + 32 * ROWS * 16;
-                        for (int item = st; item < nrows * 32; item += 128) {
+                        for (int item = st; item < nrows * 32; item += kSmx) {
                             const int c4 = item / nrows, lr = row0 + (item - c4 * nrows);
                             const int grow = sg.mblock * 128 + lr;
                             if (grow >= rows_total) continue;
