@@ -44,8 +44,8 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", default="llava7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -62,6 +62,24 @@ def measured_peaks():
             d = json.load(f)
         return float(d["hbm_gbs"]), "measured"
     return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------ rank logic
+
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity for a single process)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_gbs(bytes_per_replica_step, steps, seconds, world):
+    """Whole-job throughput of `world` independent replicas that all finished `steps` steps within `seconds`."""
+    return world * bytes_per_replica_step * steps / seconds / 1e9
 
 
 # ------------------------------------------------------------------------------------ clocks
@@ -371,12 +389,9 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     status = wl.ctx.status_poll()
 
-    t = torch.tensor([ms_total, attn_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, attn_ms = float(t[0]), float(t[1])
+    ms_total, attn_ms = max_over_ranks([ms_total, attn_ms], world, "cuda")
     kv_bytes_step = wl.kv_bytes_per_layer * L
-    value = world * kv_bytes_step * args.steps / (ms_total * 1e-3) / 1e9
+    value = whole_job_gbs(kv_bytes_step, args.steps, ms_total * 1e-3, world)
 
     # ---- end-to-end timing (host buffers in, host results out) ----
     e2e = None
@@ -385,18 +400,16 @@ def main():
         for _ in range(3):
             hs.step()
         barrier()
-        n_e2e = max(3, min(args.steps, 10))
+        n_e2e = max(3, min(args.steps, 20))
         t0 = time.perf_counter()
         for _ in range(n_e2e):
             hs.step()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * kv_bytes_step * n_e2e / float(tt[0]) / 1e9, "unit": "GB/s",
+        dt = max_over_ranks([dt], world, "cuda")[0]
+        e2e = {"value": whole_job_gbs(kv_bytes_step, n_e2e, dt, world), "unit": "GB/s",
                "h2d_bytes_per_step": hs.h2d, "d2h_bytes_per_step": hs.d2h, "steps": n_e2e,
-               "ms_per_step": 1e3 * float(tt[0]) / n_e2e}
+               "ms_per_step": 1e3 * dt / n_e2e}
 
     if rank != 0:
         if world > 1:
