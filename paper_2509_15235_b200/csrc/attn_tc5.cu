@@ -45,6 +45,7 @@
 // Every wait on an mbarrier is bounded; on a timeout the CTA records VISPEC_E_TIMEOUT, drains its own
 // copies, frees its TMEM and returns.
 #include <cuda_bf16.h>
+#include <type_traits>
 
 #include "vispec_internal.h"
 
@@ -272,7 +273,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ long long g_trace[3][64][8];
 __device__ long long g_trace_misc[16];
 __device__ int g_trace_cta = 0;
+#ifdef VISPEC_TC5_TRACE_STEPS
 #define TRACE(role, step, slot) do { if (blockIdx.x == g_trace_cta && (step) < 64) g_trace[role][step][slot] = clock64(); } while (0)
+#else
+#define TRACE(role, step, slot) do {} while (0)
+#endif
 #define TRACE_MISC(slot) do { if (blockIdx.x == g_trace_cta && threadIdx.x == 128) g_trace_misc[slot] = clock64(); } while (0)
 // Per-launch timeline in globaltimer nanoseconds: [launch][0/1] attention first start / last end, [2/3] merge.
 __device__ unsigned long long g_timeline[4096][4];
@@ -584,6 +589,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                                                               // in the epilogue: [0..255] l by (ch, lane), [256..383] m by lane
         int px = 0;                                           // phases of the pair barrier used so far
         pdl_wait();                                           // q, tree_mask and every output come after the preceding kernel
+        TRACE_MISC(4);
 
         // rejected sequences (kv_len < 0 or kv_len + N > S_max): zero output, -inf lse, status word
         {
@@ -804,6 +810,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 xm[ch * 128 + tl] = l_run;
                 if (ch == 0) xm[256 + tl] = has_o ? m_ref : -INFINITY;
                 if (!pair_sync()) { ok = false; break; }
+                TRACE_MISC(10);
                 const float l_lane = xm[tl] + xm[128 + tl];                  // l of this lane's row copy
                 float w_me = has_o ? 1.f : 0.f, w_other = 0.f, m_all = has_o ? m_ref : -INFINITY, l_all = l_lane;
                 if (PAIR) {
@@ -825,6 +832,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     } else {
                         ok = mbar_wait_warp(bar(B_XCH), seg & 1, abort_flag);
                         if (!ok) break;
+                        TRACE_MISC(11);
                         const float m_o = xm[256 + 64 + tl], l_o = xm[64 + tl] + xm[128 + 64 + tl];
                         m_all = fmaxf(m_all, m_o);
                         const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
@@ -889,66 +897,78 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     }
                     if (PAIR) mbar_arrive(bar(B_XFREE));
                 }
-                if (CL) {
-                    // ---- cluster exchange: every CTA of the unit has parked its partial in its own shared memory;
-                    // rank r merges rows [r*rp, (r+1)*rp) of all k partials and writes them out ----
-                    mbar_arrive(bar(B_EPI));
-                    bool eok = true;
-                    if (st == 0) {
-                        eok = mbar_wait(bar(B_EPI), 0, abort_flag);
-                        // signal every CTA of the cluster (this one included), whatever happened here: a peer
-                        // must never be left waiting
-                        for (int j = 0; j < ck; ++j) mbar_arrive_remote(dsmem_addr(bar(B_CL1), (uint32_t)j));
-                    }
-                    eok = mbar_wait_cluster(bar(B_CL1), 0, abort_flag) && eok;
-                    ok = __all_sync(0xffffffffu, eok);
-                    if (ok) {
-                        const int rp = (ROWS + ck - 1) / ck;
-                        const int row0 = cr * rp;
-                        const int nrows = min(rp, ROWS - row0);
-                        const uint32_t pbuf_a = base + SMEM_K, pst_a = base + SMEM_K + 32 * ROWS * 16;
-                        for (int item = st; item < nrows * 32; item += kSmx) {
-                            const int c4 = item / nrows, lr = row0 + (item - c4 * nrows);
-                            const int grow = sg.mblock * 128 + lr;
-                            if (grow >= rows_total) continue;
-                            float2 ml[8];
-                            float4 pv[8];
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                ml[j] = make_float2(-INFINITY, 0.f);
-                                pv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (j < ck) {
-                                    ml[j] = dsmem_ld2(dsmem_addr(pst_a + lr * 8, (uint32_t)j));
-                                    pv[j] = dsmem_ld4(dsmem_addr(pbuf_a + (c4 * ROWS + lr) * 16, (uint32_t)j));
-                                }
-                            }
-                            float mm = -INFINITY;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) mm = fmaxf(mm, ml[j].x);
-                            const float m_fin = (mm == -INFINITY) ? 0.f : mm;
-                            float ll = 0.f;
-                            float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const float w = exp2f(ml[j].x - m_fin);          // 0 for an empty or absent part
-                                ll += ml[j].y * w;
-                                a4.x += w * pv[j].x; a4.y += w * pv[j].y; a4.z += w * pv[j].z; a4.w += w * pv[j].w;
-                            }
-                            const float inv2 = ll > 0.f ? 1.f / ll : 0.f;
-                            const int nd = grow / G, hd = sg.kvh * G + grow % G;
-                            *reinterpret_cast<uint2*>(p.out + (((size_t)sg.b * N + nd) * p.Hq + hd) * D + c4 * 4) =
-                                make_uint2(pack_bf16(a4.x * inv2, a4.y * inv2), pack_bf16(a4.z * inv2, a4.w * inv2));
-                            if (c4 == 0 && p.lse)
-                                p.lse[((size_t)sg.b * p.Hq + hd) * N + nd] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
-                        }
-                    }
-                    if (!ok) break;
-                }
+                if (CL) TRACE_MISC(12);
                 tc_fence_before();        // the next segment's first product overwrites O
                 TRACE_MISC(7);
                 ++seg;
             }
         }
+    }
+
+    if (CL) {
+        // ---- cluster exchange: every CTA of the unit has parked its partial (O, m, l) in its own shared memory.
+        // All threads of the cluster meet at the hardware cluster barrier (the warps that finished early wait
+        // there without polling); then rank r merges rows [r*rp, (r+1)*rp) of all k partials through distributed
+        // shared memory and writes them out. ----
+        __syncwarp();
+        cluster_sync_all();
+        TRACE_MISC(13);
+        if (warp >= 4 && !*abort_flag) {
+        const int rp = (ROWS + ck - 1) / ck;
+        const int row0 = cr * rp;
+        const int nrows = min(rp, ROWS - row0);
+        const uint32_t pbuf_a = base + SMEM_K, pst_a = base + SMEM_K + 32 * ROWS * 16;
+        // IT items (row, column quad) at a time per thread, all loads of all KM pieces issued before the first use
+        auto merge_items = [&](auto km_tag, auto it_tag) {
+            constexpr int KM = decltype(km_tag)::value, IT = decltype(it_tag)::value;
+            for (int item0 = tid - 128; item0 < nrows * 32; item0 += kSmx * IT) {
+                float2 ml[IT][KM];
+                float4 pv[IT][KM];
+                int c4s[IT], grows[IT];
+#pragma unroll
+                for (int e = 0; e < IT; ++e) {
+                    const int item = item0 + e * kSmx;
+                    const int c4 = item / nrows, lr = row0 + (item - c4 * nrows);
+                    c4s[e] = c4;
+                    grows[e] = (item < nrows * 32) ? cl_seg.mblock * 128 + lr : rows_total;
+#pragma unroll
+                    for (int j = 0; j < KM; ++j) {
+                        ml[e][j] = make_float2(-INFINITY, 0.f);
+                        pv[e][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (j < ck && grows[e] < rows_total) {
+                            ml[e][j] = dsmem_ld2(dsmem_addr(pst_a + lr * 8, (uint32_t)j));
+                            pv[e][j] = dsmem_ld4(dsmem_addr(pbuf_a + (c4 * ROWS + lr) * 16, (uint32_t)j));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < IT; ++e) {
+                    if (grows[e] >= rows_total) continue;
+                    float mm = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < KM; ++j) mm = fmaxf(mm, ml[e][j].x);
+                    const float m_fin = (mm == -INFINITY) ? 0.f : mm;
+                    float ll = 0.f;
+                    float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int j = 0; j < KM; ++j) {
+                        const float w = exp2f(ml[e][j].x - m_fin);          // 0 for an empty or absent part
+                        ll += ml[e][j].y * w;
+                        a4.x += w * pv[e][j].x; a4.y += w * pv[e][j].y; a4.z += w * pv[e][j].z; a4.w += w * pv[e][j].w;
+                    }
+                    const float inv2 = ll > 0.f ? 1.f / ll : 0.f;
+                    const int nd = grows[e] / G, hd = cl_seg.kvh * G + grows[e] % G;
+                    *reinterpret_cast<uint2*>(p.out + (((size_t)cl_seg.b * N + nd) * p.Hq + hd) * D + c4s[e] * 4) =
+                        make_uint2(pack_bf16(a4.x * inv2, a4.y * inv2), pack_bf16(a4.z * inv2, a4.w * inv2));
+                    if (c4s[e] == 0 && p.lse)
+                        p.lse[((size_t)cl_seg.b * p.Hq + hd) * N + nd] = ll > 0.f ? (mm + log2f(ll)) * 0.6931471805599453f : -INFINITY;
+                }
+            }
+        };
+        if (ck <= 4) merge_items(std::integral_constant<int, 4>{}, std::integral_constant<int, 2>{});
+        else merge_items(std::integral_constant<int, 8>{}, std::integral_constant<int, 1>{});
+        }
+        TRACE_MISC(14);
     }
 
     // ---- tear-down: everyone meets, TMEM goes back ----
