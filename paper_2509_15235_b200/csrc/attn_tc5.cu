@@ -128,10 +128,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+// The K/V tiles are read once per call: they are marked evict-first in L2 so that the stream does not push out
+// what is read again soon (q, masks, partial results, the next kernels' operands).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, uint64_t pol) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -478,6 +485,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0 && active) {
+            const uint64_t pol = l2_evict_first_policy();
             bool waited = !p.early;
             int it = 0, nk = 0, nv = 0;          // steps started; K / V stages issued
             bool ok = true;
@@ -493,14 +501,14 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     if (!mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag)) { ok = false; break; }
                     TRACE(0, it, 1);
                     mbar_expect_tx(bar(B_KFULL + sk), STAGE_BYTES);
-                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES, &k_map, bar(B_KFULL + sk), 0, tok, bh);
-                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES, &k_map, bar(B_KFULL + sk), 64, tok, bh);
+                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES, &k_map, bar(B_KFULL + sk), 0, tok, bh, pol);
+                    tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES, &k_map, bar(B_KFULL + sk), 64, tok, bh, pol);
                     ++nk;
                     if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { ok = false; break; }
                     TRACE(0, it, 2);
                     mbar_expect_tx(bar(B_VFULL + sv), STAGE_BYTES);
-                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES, &v_map, bar(B_VFULL + sv), 0, tok, bh);
-                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES, &v_map, bar(B_VFULL + sv), 64, tok, bh);
+                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES, &v_map, bar(B_VFULL + sv), 0, tok, bh, pol);
+                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES, &v_map, bar(B_VFULL + sv), 64, tok, bh, pol);
                     ++nv;
                 }
             }
