@@ -45,7 +45,6 @@
 // Every wait on an mbarrier is bounded; on a timeout the CTA records VISPEC_E_TIMEOUT, drains its own
 // copies, frees its TMEM and returns.
 #include <cuda_bf16.h>
-#include <cstdlib>
 #include <type_traits>
 
 #include "vispec_internal.h"
@@ -997,8 +996,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     CTA_T(1);
 }
 
-#include "attn_tc5_tform.cuh"
-
 // Merge of the partials of every unit that more than one CTA worked on.  Grid (unit, 2 * group of 32 rows +
 // half of the columns), 4 warps; lane <-> row, a warp sums 16 output columns over the unit's segments.
 // The blocks are small so that they fit beside a resident attention CTA: they are launched early
@@ -1148,8 +1145,7 @@ static int query_max_clusters(bool pair, int k) {
     attr[0].val.clusterDim.x = k; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int n = 0;
-    if (pair) cfg.dynamicSmemBytes = T_SMEM_TOTAL;
-    cudaError_t e = pair ? cudaOccupancyMaxActiveClusters(&n, attn_tc5t_kernel<true>, &cfg)
+    cudaError_t e = pair ? cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<true, true>, &cfg)
                          : cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<false, true>, &cfg);
     if (e != cudaSuccess) { cudaGetLastError(); return 0; }
     return n;
@@ -1188,10 +1184,6 @@ cudaError_t init_attn_tc5() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc5_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc5t_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_TOTAL);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc5t_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_TOTAL);
-    if (e != cudaSuccess) return e;
     for (int k = 1; k <= 8; ++k) { g_max_clusters[0][k] = query_max_clusters(false, k); g_max_clusters[1][k] = query_max_clusters(true, k); }
     // The merge blocks must be able to join an SM that an attention CTA has configured for maximum shared memory.
     e = cudaFuncSetAttribute(attn_tc5_merge_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -1226,23 +1218,6 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     p.trace_idx = 0;
 #endif
     cudaError_t err;
-    static const bool row_major_small = [] { const char* e = getenv("VISPEC_TC5_ROWMAJOR"); return e && e[0] == '1'; }();
-    if (pair && !row_major_small) {
-        // at most 64 rows per unit: the transposed form
-        if (ck > 0) {
-            err = launch_pdl(attn_tc5t_kernel<true>, dim3(grid), dim3(kThreads), T_SMEM_TOTAL, st, ck, *a.k_map, *a.v_map, p);
-            if (err != cudaSuccess) return err;
-            ++*n_launches;
-            return cudaSuccess;
-        }
-        err = launch_pdl(attn_tc5t_kernel<false>, dim3(grid), dim3(kThreads), T_SMEM_TOTAL, st, 0, *a.k_map, *a.v_map, p);
-        if (err != cudaSuccess) return err;
-        ++*n_launches;
-        err = launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p);
-        if (err != cudaSuccess) return err;
-        ++*n_launches;
-        return cudaSuccess;
-    }
     if (ck > 0) {
         // cluster form: the CTAs of a unit merge their partials through distributed shared memory; one launch
         err = pair ? launch_pdl(attn_tc5_kernel<true, true>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, ck, *a.k_map, *a.v_map, p)
