@@ -51,6 +51,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
+    ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context: 0 automatic, 1 partials + merge kernel, 2 clusters")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying graphs")
     return ap.parse_args()
 
@@ -353,6 +354,9 @@ def main():
 
     tree, per_layer = build_host_inputs(cfg, args.layers if args.layers > 0 else cfg.layers)
     wl = DeviceWorkload(cfg, tree, per_layer, local)
+    if args.split_form:
+        from paper_2509_15235_b200 import binding
+        wl.ctx.ctx_set_option(binding.OPT_SPLIT_FORM, args.split_form)
     L = wl.L
 
     def barrier():

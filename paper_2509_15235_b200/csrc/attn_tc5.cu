@@ -45,6 +45,8 @@
 // Every wait on an mbarrier is bounded; on a timeout the CTA records VISPEC_E_TIMEOUT, drains its own
 // copies, frees its TMEM and returns.
 #include <cuda_bf16.h>
+#include <cstdio>
+#include <cstdlib>
 #include <type_traits>
 
 #include "vispec_internal.h"
@@ -77,7 +79,7 @@ constexpr long long kWaitCycles = 1500000000LL;                // ~0.8 s at 1.9 
 enum { B_KFULL = 0, B_KEMPTY = B_KFULL + NSK, B_VFULL = B_KEMPTY + NSK, B_VEMPTY = B_VFULL + NSV,
        B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2,
        B_QFULL = B_PVDONE + 2, B_PAIRX = B_QFULL + 1, B_XCH = B_PAIRX + 4, B_XFREE = B_XCH + 1,
-       B_EPI = B_XFREE + 1, B_CL1 = B_EPI + 1, B_COUNT = B_CL1 + 1 };
+       B_COUNT = B_XFREE + 1 };
 static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block too small");
 
 // The schedule every CTA (and the merge kernel) derives from kv_len.
@@ -156,33 +158,11 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
     uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank)); return r;
 }
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
-}
 __device__ __forceinline__ float4 dsmem_ld4(uint32_t a) {
     float4 v; asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory"); return v;
 }
 __device__ __forceinline__ float2 dsmem_ld2(uint32_t a) {
     float2 v; asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a) : "memory"); return v;
-}
-// Bounded wait like mbar_wait, acquiring at cluster scope (the arrivals come from other CTAs of the cluster).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-        if ((it & 63) == 63) {
-            if (*abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitCycles) { *abort_flag = 1; return false; }
-        }
-    }
 }
 // Programmatic dependent launch: let the next kernel in the stream be scheduled / wait for the previous one.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -291,8 +271,8 @@ __device__ unsigned long long g_timeline[4096][4];
 __device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 __device__ unsigned long long g_cta_times[256][4];
 #define CTA_T(k) do { if (threadIdx.x == 0 && blockIdx.x < 256) g_cta_times[blockIdx.x][k] = gtimer(); } while (0)
-#define TL_START(idx, k) do { if (threadIdx.x == 0 && (idx) < 4096) atomicMin(&g_timeline[idx][k], gtimer()); } while (0)
-#define TL_END(idx, k) do { if (threadIdx.x == 0 && (idx) < 4096) atomicMax(&g_timeline[idx][k], gtimer()); } while (0)
+#define TL_START(idx, k) do { if ((idx) < 4096) atomicMin(&g_timeline[idx][k], gtimer()); } while (0)
+#define TL_END(idx, k) do { if ((idx) < 4096) atomicMax(&g_timeline[idx][k], gtimer()); } while (0)
 #else
 #define CTA_T(k) do {} while (0)
 #define TL_START(idx, k) do {} while (0)
@@ -409,7 +389,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
     extern __shared__ __align__(1024) unsigned char sm[];
     TRACE_MISC(0);
-    TL_START(p.trace_idx, 0);
+    if (threadIdx.x == 0) TL_START(p.trace_idx, 0);
     CTA_T(0);
     const uint32_t base = smem_u32(sm);
     if (base & 1023u) {
@@ -438,8 +418,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         for (int i = 0; i < 4; ++i) mbar_init(bar(B_PAIRX + i), 64);
         mbar_init(bar(B_QFULL), kSmx);
         mbar_init(bar(B_XCH), 128); mbar_init(bar(B_XFREE), 128);
-        mbar_init(bar(B_EPI), kSmx);
-        mbar_init(bar(B_CL1), CL ? cluster_size() : 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -453,7 +431,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     TRACE_MISC(1);
     tc_fence_before();
     __syncthreads();
-    if (CL) cluster_sync_all();          // every CTA's barriers exist before a peer can signal them
     tc_fence_after();
     TRACE_MISC(2);
 
@@ -597,6 +574,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                                                               // in the epilogue: [0..255] l by (ch, lane), [256..383] m by lane
         int px = 0;                                           // phases of the pair barrier used so far
         pdl_wait();                                           // q, tree_mask and every output come after the preceding kernel
+        if (tid == 128) { TL_START(p.trace_idx, 2); TL_END(p.trace_idx, 3); }
         TRACE_MISC(4);
 
         // rejected sequences (kv_len < 0 or kv_len + N > S_max): zero output, -inf lse, status word
@@ -992,7 +970,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
     }
     if (tid == 0 && *abort_flag) atomicCAS(p.status, 0, (int)VISPEC_E_TIMEOUT);
-    TL_END(p.trace_idx, 1);
+    if (threadIdx.x == 0) TL_END(p.trace_idx, 1);
     CTA_T(1);
 }
 
@@ -1125,7 +1103,7 @@ extern "C" int vispec_debug_timeline(unsigned long long* host, int reset) {
     if (reset) {
         g_trace_launch = 0;
         static unsigned long long init[4096][4];
-        for (int i = 0; i < 4096; ++i) { init[i][0] = ~0ull; init[i][1] = 0; init[i][2] = 0; init[i][3] = ~0ull; }
+        for (int i = 0; i < 4096; ++i) { init[i][0] = ~0ull; init[i][1] = 0; init[i][2] = ~0ull; init[i][3] = 0; }
         return cudaMemcpyToSymbol(g_timeline, init, sizeof(init)) == cudaSuccess ? 0 : -1;
     }
     return cudaMemcpyFromSymbol(host, g_timeline, sizeof(g_timeline)) == cudaSuccess ? 0 : -1;
@@ -1185,6 +1163,7 @@ cudaError_t init_attn_tc5() {
     e = cudaFuncSetAttribute(attn_tc5_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
     if (e != cudaSuccess) return e;
     for (int k = 1; k <= 8; ++k) { g_max_clusters[0][k] = query_max_clusters(false, k); g_max_clusters[1][k] = query_max_clusters(true, k); }
+    if (getenv("VISPEC_DEBUG")) for (int k = 1; k <= 8; ++k) fprintf(stderr, "vispec: cluster size %d: %d (rows > 64) / %d (rows <= 64) co-resident clusters\n", k, g_max_clusters[0][k], g_max_clusters[1][k]);
     // The merge blocks must be able to join an SM that an attention CTA has configured for maximum shared memory.
     e = cudaFuncSetAttribute(attn_tc5_merge_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
