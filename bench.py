@@ -438,7 +438,7 @@ def main():
         "pct_of_8TBs": 100.0 * achieved / 8000.0,
         "status_word": status,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": "vispec_tree_verify_attn (main kernel + merge)",
+                     "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 3) // L} kernel launch(es) per call)",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)},
         "clocks": clocks,
         "gpu_launches": int(launches),

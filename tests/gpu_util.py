@@ -29,7 +29,7 @@ def u64_host(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().numpy().view(np.uint64)
 
 
-def run_attn(q, k, v, kv_len, mask, scale, want_lse=True, B_max=None, N_max=None, split_form=0):
+def run_attn(q, k, v, kv_len, mask, scale, want_lse=True, B_max=None, N_max=None, split_form=0, early_prefetch=None):
     """One attention call through the C ABI.  Inputs are numpy (bf16 bits / int32 / uint64).
     Returns (out float32 [B,N,Hq,D], lse float32 [B,Hq,N] or None, status word)."""
     B, N, Hq, D = q.shape
@@ -37,6 +37,8 @@ def run_attn(q, k, v, kv_len, mask, scale, want_lse=True, B_max=None, N_max=None
     ctx = binding.VerifyContext(B_max or max(B, 1), N_max or N, Hq, Hkv, D, S_max, 1)
     if split_form:
         ctx.ctx_set_option(binding.OPT_SPLIT_FORM, split_form)
+    if early_prefetch is not None:
+        ctx.ctx_set_option(binding.OPT_EARLY_PREFETCH, int(early_prefetch))
     kd, vd = bf16_dev(k), bf16_dev(v)
     ctx.cache_register(0, kd, vd)
     qd = bf16_dev(q)

@@ -209,3 +209,29 @@ def test_long_response_sweep_cells(gu, name):
     want, want_lse = oracle.tree_attn(q[:, :, hs], k[:, kvh:kvh + 1], v[:, kvh:kvh + 1], kv_len, mask, scale)
     assert np.abs(out[:, :, hs] - want).max() <= TOL
     assert np.abs(lse[:, hs] - want_lse).max() <= LSE_TOL
+
+
+def test_options_and_fallbacks_give_the_same_attention(gu):
+    """Early prefix prefetch off, more sequences than the tensor-core kernel takes per call (generic kernel),
+    and a non-positive scale (generic kernel: the maximum no longer commutes with the scale)."""
+    from paper_2509_15235_b200 import binding
+    rng = np.random.Generator(np.random.Philox(2024))
+    Hq, Hkv, D, N, S_max = 4, 2, 128, 12, 384
+    for B, scale, early in ((2, 0.09, 0), (33, 0.09, None), (2, 0.0, None), (2, -0.05, None)):
+        q = synth.normal_bf16((B, N, Hq, D), 71 + B); k = synth.normal_bf16((B, Hkv, S_max, D), 72 + B)
+        v = synth.normal_bf16((B, Hkv, S_max, D), 73 + B)
+        kv_len = rng.integers(0, S_max - N, size=B).astype(np.int32)
+        parents = np.stack([synth.draw_tree(N, 4, 3, rng) for _ in range(B)])
+        mask, _, _ = oracle.tree_mask(parents)
+        out, lse, status = gu.run_attn(q, k, v, kv_len, mask, scale, early_prefetch=early)
+        want, want_lse = oracle.tree_attn(q, k, v, kv_len, mask, scale)
+        assert status == 0
+        assert np.abs(out - want).max() <= TOL
+        assert np.abs(lse - want_lse).max() <= LSE_TOL
+    ctx = binding.VerifyContext(1, 8, 2, 2, 64, 128, 1)
+    with pytest.raises(binding.VispecError) as e:
+        ctx.ctx_set_option(99, 1)
+    assert e.value.code == -5
+    with pytest.raises(binding.VispecError) as e:
+        ctx.ctx_set_option(binding.OPT_SPLIT_FORM, 7)
+    assert e.value.code == -4
