@@ -1,21 +1,26 @@
 // Tree-verification attention for sm_100a (D = 128): TMA-staged K/V tiles, tcgen05 tensor-core products
-// with every accumulator AND both A operands in TMEM, fp32 online softmax (Eq. 1 restricted to prefix +
-// ancestors), work split evenly over the SMs.
+// with fp32 accumulators in TMEM, fp32 online softmax (Eq. 1 restricted to prefix + ancestors), work split
+// over the SMs.
 //
-// Work.  A *unit* is (sequence, kv head, block of query rows); it needs ceil((S+N)/128) *steps*, one per
-// 128 cached tokens.  All steps of all units, in the order (sequence, kv head, row block, step), form one
-// line of T steps that is cut into equal ranges, one per CTA (at most one CTA per SM; when the units are fewer
-// than the SMs the CTA count is a multiple of the unit count, so that equally long units are cut into whole
-// CTAs).  A CTA therefore runs a
-// few *segments*: the tail of one unit, whole units, the head of another.  A segment that covers its
-// whole unit writes the final bf16 output; any other writes an unnormalised partial (O, m, l) into one of
-// the CTA's two slots (first segment -> slot 2c, a later one -> slot 2c+1) and a second, small kernel merges
-// the partials of each unit.  Both kernels derive the same schedule from kv_len on the device, so the
-// host never reads lengths.
+// Work.  A *unit* is (sequence, kv head, block of <= 128 query rows, rows ordered node-major so that all heads
+// and nodes of a head group share every K/V tile); it needs ceil((S+N)/128) *steps*, one per 128 cached
+// tokens.  Two ways to spread the units over the CTAs (at most one CTA per SM):
+//   cluster form     one thread-block cluster of k <= 8 CTAs per unit; the CTA of rank r takes the r-th of k
+//                    equal parts of the unit's steps and parks its unnormalised partial (O, m, l) in its own
+//                    shared memory; after a hardware cluster barrier rank r merges rows [r*rows/k, ...) of all
+//                    k partials through distributed shared memory and writes them out.  One launch.
+//   even split       all steps of all units, in the order (sequence, kv head, row block, step), form one line
+//                    of T steps cut into equal ranges, one per CTA (the CTA count is a multiple of the unit
+//                    count when the units are fewer than the SMs, so that equally long units are cut into
+//                    whole CTAs).  A CTA runs a few *segments*: the tail of one unit, whole units, the head of
+//                    another.  A segment that covers its whole unit writes the final bf16 output; any other
+//                    writes a partial into one of the CTA's two slots (first segment -> slot 2c, a later one
+//                    -> slot 2c+1) and a second, small kernel merges the partials of each unit.
+// Both kernels derive the schedule from kv_len on the device, so the host never reads lengths.
 //
 // Inside a CTA the 12 warps are specialised:
-//   warp 0     TMA producer: K ring and V ring of 128-token stages (32 KB each, 128-byte swizzle); it runs
-//              ahead across segment boundaries
+//   warp 0     TMA producer: K ring and V ring of 128-token stages (3 x 32 KB each, 128-byte swizzle, evict-first
+//              in L2); it runs ahead across segment boundaries
 //   warp 1     issuer (one thread) of S = Q K^T as 128x128x16 tcgen05.mma; owns the TMEM allocation
 //   warp 2     issuer (one thread) of O += P V; the two chains wait on different barriers, so each has its own
 //              thread and neither's waits delay the other's instructions
@@ -30,20 +35,21 @@
 // product of step u-1 run while step u is in the softmax.
 //
 // Two row layouts share the code:
-//   FULL  (G*N > 64):  lane r holds query row r of the block; a thread handles all 128 tokens of a step.
+//   FULL  (G*N > 64):  lane r holds query row r of the block.
 //   PAIR  (G*N <= 64): the <= 64 query rows are duplicated, lanes 0-63 take tokens 0-63 of each step and
 //                      lanes 64-127 tokens 64-127 (P is block-diagonal); the two halves keep independent
 //                      softmax states and are merged once per segment through shared memory.
 // The running maximum is only moved when a tile exceeds it by more than 2^8 (O and l share the reference, so
 // the result is exact either way); O is therefore re-scaled in TMEM rarely.
 //
-// Programmatic dependent launch: both kernels are launched with programmatic stream serialisation.  The
+// Programmatic dependent launch: every launch carries the programmatic stream serialisation attribute.  The
 // attention kernel reads kv_len and (when early prefetch is on) streams K/V tiles that lie wholly inside the
 // committed prefix before it waits for the preceding kernel; q, tree_mask, the tree's own K/V rows and every
 // write come after that wait.
 //
 // Every wait on an mbarrier is bounded; on a timeout the CTA records VISPEC_E_TIMEOUT, drains its own
-// copies, frees its TMEM and returns.
+// copies, frees its TMEM and returns.  The cluster form's two hardware cluster barriers are reached by every
+// thread of every CTA of the cluster (all other waits being bounded), so they end.
 #include <cuda_bf16.h>
 #include <cstdio>
 #include <cstdlib>
