@@ -203,6 +203,18 @@ int vispec_kv_compact(vispec_ctx* ctx, int layer_begin, int layer_end, const int
                       const int32_t* accept_len, const int32_t* kv_len, int32_t* kv_len_out,
                       int B, int N, void* stream);
 
+/* Acceptance and commit in one launch: the result of vispec_accept followed by vispec_kv_compact over the
+ * registered layers [layer_begin, layer_end) (Sec. 3.1 acceptance at temperature 0, then the App. A commit of
+ * the accepted path's K/V rows), without the second launch and the dependency between the two.  Arguments,
+ * outputs (path, accept_len, bonus, kv_len_out = S + accept_len; kv_len_out may be NULL and must not alias
+ * kv_len) and status-word behaviour are those of the two calls: an invalid tree commits the root only
+ * (VISPEC_E_BAD_TREE), a sequence with kv_len < 0 or kv_len + N > S_max gets its acceptance outputs but no
+ * commit (VISPEC_E_RANGE).  With layer_begin == layer_end only the acceptance runs.
+ * Host errors: E_NULL, E_SHAPE, E_RANGE (layers), E_UNREGISTERED. */
+int vispec_accept_commit(vispec_ctx* ctx, int layer_begin, int layer_end, const int32_t* draft_ids,
+                         const int32_t* target_ids, const int32_t* parents, const int32_t* kv_len, int B, int N,
+                         int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, void* stream);
+
 /* Read and clear the device status word (synchronises `stream`; not a hot call).
  * `*code` (host) receives VISPEC_OK or the first asynchronous error recorded since the last poll. */
 int vispec_status_poll(vispec_ctx* ctx, int* code /*host*/, void* stream);

@@ -59,16 +59,12 @@ cudaError_t launch_tree_mask(const int32_t* parents, int B, int N, uint64_t* mas
 // reachable node (smallest index among equals), found with a shuffle max-reduction on the key
 // depth*256 + (255 - index).
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(32)
-accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ target,
-              const int32_t* __restrict__ parents, int N, int32_t* __restrict__ path,
-              int32_t* __restrict__ accept_len, int32_t* __restrict__ bonus, int* status) {
-    __shared__ int32_t par[VISPEC_MAX_TREE_NODES];
-    __shared__ int32_t tgt[VISPEC_MAX_TREE_NODES];
-    const int b = blockIdx.x, lane = threadIdx.x;
-    const size_t base = (size_t)b * N;
-    for (int i = lane; i < N; i += 32) { par[i] = parents[base + i]; tgt[i] = target[base + i]; }
-    __syncwarp();
+// One warp decides one sequence.  par / tgt are shared-memory copies of the sequence's parents and target ids
+// (filled by the caller, visible to the warp).  Returns (warp-uniform) the accepted length; `path_out[0..N)`
+// (any memory the warp can write) receives the path padded with -1, `*bonus_out` the bonus token (lane 0).
+__device__ int accept_warp(const int32_t* __restrict__ draft_row, const int32_t* par, const int32_t* tgt, int N,
+                           int32_t* path_out, int32_t* bonus_out, int* status) {
+    const int lane = threadIdx.x & 31;
     // validity of the whole tree (every link must point to an earlier node)
     bool tree_ok = true;
     for (int i = lane; i < N; i += 32) tree_ok &= (i == 0) ? (par[0] == -1) : (par[i] >= 0 && par[i] < i);
@@ -79,7 +75,7 @@ accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ tar
     for (int w = 0; w < 4; ++w) {
         const int i = w * 32 + lane;
         bool m = false;
-        if (tree_ok && i < N) m = (i == 0) || (draft[base + i] == tgt[par[i]]);
+        if (tree_ok && i < N) m = (i == 0) || (draft_row[i] == tgt[par[i]]);
         matched[w] = __ballot_sync(0xffffffffu, m);
     }
     int best_key = -1;
@@ -103,13 +99,27 @@ accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ tar
     for (int off = 16; off > 0; off >>= 1) best_key = max(best_key, __shfl_xor_sync(0xffffffffu, best_key, off));
     const int best_depth = best_key >> 8;
     const int best = 255 - (best_key & 255);
-    for (int k = lane; k < N; k += 32) if (k > best_depth) path[base + k] = -1;
+    for (int k = lane; k < N; k += 32) if (k > best_depth) path_out[k] = -1;
     if (lane == 0) {
         int a = best;
-        for (int k = best_depth; k >= 0; --k) { path[base + k] = a; a = (a == 0) ? 0 : par[a]; }
-        accept_len[b] = best_depth + 1;
-        bonus[b] = tgt[best];
+        for (int k = best_depth; k >= 0; --k) { path_out[k] = a; a = (a == 0) ? 0 : par[a]; }
+        *bonus_out = tgt[best];
     }
+    return best_depth + 1;
+}
+
+__global__ void __launch_bounds__(32)
+accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ target,
+              const int32_t* __restrict__ parents, int N, int32_t* __restrict__ path,
+              int32_t* __restrict__ accept_len, int32_t* __restrict__ bonus, int* status) {
+    __shared__ int32_t par[VISPEC_MAX_TREE_NODES];
+    __shared__ int32_t tgt[VISPEC_MAX_TREE_NODES];
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const size_t base = (size_t)b * N;
+    for (int i = lane; i < N; i += 32) { par[i] = parents[base + i]; tgt[i] = target[base + i]; }
+    __syncwarp();
+    const int len = accept_warp(draft + base, par, tgt, N, path + base, bonus + b, status);
+    if (lane == 0) accept_len[b] = len;
 }
 
 cudaError_t launch_accept(const int32_t* draft, const int32_t* target, const int32_t* parents, int B,
@@ -184,6 +194,80 @@ cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int laye
     dim3 grid(Hkv, B, layer_end - layer_begin);
     kv_compact_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, path, accept_len, kv_len, kv_len_out,
                                             N, Hkv, D, S_max, status);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Acceptance and commit in one launch (Sec. 3.1 acceptance followed by the App. A commit): every block
+// (layer, sequence, kv head) repeats the cheap acceptance of its sequence in its first warp, keeps the path
+// in shared memory and then moves its head's rows exactly as kv_compact_kernel does; the block of the first
+// layer and head also writes path, accept_len, bonus and kv_len_out.  Saves a launch and a dependency per
+// decoding cycle.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+accept_commit_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const int32_t* __restrict__ draft,
+                     const int32_t* __restrict__ target, const int32_t* __restrict__ parents,
+                     const int32_t* __restrict__ kv_len, int32_t* __restrict__ path, int32_t* __restrict__ accept_len,
+                     int32_t* __restrict__ bonus, int32_t* __restrict__ kv_len_out, int N, int Hkv, int D, int S_max,
+                     int* status) {
+    __shared__ uint4 stage[2][kCompactRows][16];
+    __shared__ int32_t par[VISPEC_MAX_TREE_NODES];
+    __shared__ int32_t tgt[VISPEC_MAX_TREE_NODES];
+    __shared__ int32_t spath[VISPEC_MAX_TREE_NODES];
+    __shared__ int32_t s_len, s_bonus;
+    const int layer = layer_begin + blockIdx.z, b = blockIdx.y, h = blockIdx.x;
+    const size_t rb = (size_t)b * N;
+    for (int i = threadIdx.x; i < N; i += 256) { par[i] = parents[rb + i]; tgt[i] = target[rb + i]; }
+    __syncthreads();
+    const bool writer = (blockIdx.x == 0 && blockIdx.z == 0);
+    if (threadIdx.x < 32) {
+        const int len = accept_warp(draft + rb, par, tgt, N, spath, &s_bonus, writer ? status : nullptr);
+        if (threadIdx.x == 0) s_len = len;
+    }
+    __syncthreads();
+    const int S = kv_len[b], L = s_len;
+    if (writer) {
+        for (int i = threadIdx.x; i < N; i += 256) path[rb + i] = spath[i];
+        if (threadIdx.x == 0) { accept_len[b] = L; bonus[b] = s_bonus; }
+    }
+    const bool ok = (S >= 0 && S + N <= S_max);
+    if (!ok) {
+        if (threadIdx.x == 0 && writer) record_status(status, VISPEC_E_RANGE);
+        return;   // kv_len_out[b] keeps its previous value for a rejected sequence
+    }
+    const int chunks = D / 8;
+    const int tensor = threadIdx.x >> 7;             // 0: K, 1: V
+    const int r = (threadIdx.x & 127) >> 3;          // row of the pass, 0..15
+    const int c0 = threadIdx.x & 7;                  // this thread moves chunks c0 and c0 + 8
+    uint4* base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]) +
+                  ((size_t)b * Hkv + h) * (size_t)S_max * chunks;
+    for (int k0 = 0; k0 < L; k0 += kCompactRows) {
+        const int k = k0 + r;
+        const int s = (k < L && spath[k] != k) ? spath[k] : -1;     // -1: nothing to move
+        if (s >= 0) {
+            const uint4* src = base + (size_t)(S + s) * chunks;
+            if (c0 < chunks) stage[tensor][r][c0] = src[c0];
+            if (c0 + 8 < chunks) stage[tensor][r][c0 + 8] = src[c0 + 8];
+        }
+        __syncthreads();
+        if (s >= 0) {
+            uint4* dst = base + (size_t)(S + k) * chunks;
+            if (c0 < chunks) dst[c0] = stage[tensor][r][c0];
+            if (c0 + 8 < chunks) dst[c0 + 8] = stage[tensor][r][c0 + 8];
+        }
+        __syncthreads();
+    }
+    if (kv_len_out && writer && threadIdx.x == 0) kv_len_out[b] = S + L;
+}
+
+cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int layer_end, const int32_t* draft,
+                                 const int32_t* target, const int32_t* parents, const int32_t* kv_len,
+                                 int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, int B, int N,
+                                 int Hkv, int D, int S_max, int* status, cudaStream_t st) {
+    if (B == 0 || layer_end <= layer_begin) return cudaSuccess;
+    dim3 grid(Hkv, B, layer_end - layer_begin);
+    accept_commit_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, draft, target, parents, kv_len, path,
+                                               accept_len, bonus, kv_len_out, N, Hkv, D, S_max, status);
     return cudaGetLastError();
 }
 

@@ -229,6 +229,30 @@ int vispec_kv_compact(vispec_ctx* c, int layer_begin, int layer_end, const int32
     return VISPEC_OK;
 }
 
+int vispec_accept_commit(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* draft_ids,
+                         const int32_t* target_ids, const int32_t* parents, const int32_t* kv_len, int B, int N,
+                         int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, void* stream) {
+    if (!c || !draft_ids || !target_ids || !parents || !kv_len || !path || !accept_len || !bonus) return VISPEC_E_NULL;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
+    if (layer_begin < 0 || layer_end > s.layers || layer_begin > layer_end) return VISPEC_E_RANGE;
+    if (kv_len_out == kv_len) return VISPEC_E_SHAPE;
+    for (int l = layer_begin; l < layer_end; ++l)
+        if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
+    if (layer_end == layer_begin) {
+        // nothing to commit: plain acceptance
+        if (launch_accept(draft_ids, target_ids, parents, B, N, path, accept_len, bonus, c->d_status,
+                          (cudaStream_t)stream) != cudaSuccess)
+            return VISPEC_E_CUDA;
+    } else if (launch_accept_commit(c->d_cache_ptrs, layer_begin, layer_end, draft_ids, target_ids, parents, kv_len,
+                                    path, accept_len, bonus, kv_len_out, B, N, s.Hkv, s.D, s.S_max, c->d_status,
+                                    (cudaStream_t)stream) != cudaSuccess) {
+        return VISPEC_E_CUDA;
+    }
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
 int vispec_status_poll(vispec_ctx* c, int* code, void* stream) {
     if (!c || !code) return VISPEC_E_NULL;
     cudaStream_t st = (cudaStream_t)stream;

@@ -45,6 +45,11 @@ cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int laye
                               int32_t* kv_len_out, int B, int N, int Hkv, int D, int S_max, int* status,
                               cudaStream_t st);
 
+cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int layer_end, const int32_t* draft,
+                                 const int32_t* target, const int32_t* parents, const int32_t* kv_len,
+                                 int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, int B, int N,
+                                 int Hkv, int D, int S_max, int* status, cudaStream_t st);
+
 struct AttnArgs {
     const void* q; const void* k; const void* v;
     const int32_t* kv_len; const uint64_t* mask;

@@ -235,3 +235,26 @@ def test_options_and_fallbacks_give_the_same_attention(gu):
     with pytest.raises(binding.VispecError) as e:
         ctx.ctx_set_option(binding.OPT_SPLIT_FORM, 7)
     assert e.value.code == -4
+
+
+def test_redundant_image_keys_stress_the_softmax(gu):
+    """Sec. 4.1 of the paper: image tokens are highly redundant, identical tokens get identical scores (Eq. 2)
+    and their softmax mass is spread evenly (Eq. 3-4).  1296 identical 'image' keys followed by ordinary text
+    keys: a huge, flat block of probability mass, against the oracle; and with every key identical the output
+    must be the mean of the visible V rows (Eq. 4), checked directly."""
+    B, N, Hq, Hkv, D, S, S_max = 1, 16, 4, 2, 128, 1500, 1664
+    rng = np.random.Generator(np.random.Philox(404))
+    q = synth.normal_bf16((B, N, Hq, D), 81); k = synth.normal_bf16((B, Hkv, S_max, D), 82)
+    v = synth.normal_bf16((B, Hkv, S_max, D), 83)
+    k[:, :, :1296] = k[:, :, :1]                       # the image span repeats one key per head
+    parents = synth.draw_tree(N, 4, 3, rng)[None]
+    mask, _, _ = oracle.tree_mask(parents)
+    _check(gu, q, k, v, np.array([S], dtype=np.int32), mask, 1 / math.sqrt(D))
+    k[:, :, :] = k[:, :, :1]                           # every key identical: weights are uniform over the visible set
+    out, lse, status = gu.run_attn(q, k, v, [S], mask, 1 / math.sqrt(D))
+    assert status == 0
+    vf = synth.bf16_bits_to_f32(v).astype(np.float64)
+    for i in range(N):
+        vis = list(range(S)) + [S + t for t in range(N) if (int(mask[0, i, 0]) >> t) & 1]
+        for h in range(Hq):
+            assert np.abs(out[0, i, h] - vf[0, h // (Hq // Hkv), vis].mean(axis=0)).max() <= TOL

@@ -211,3 +211,67 @@ def test_compact_out_of_range_sequence_is_skipped_with_status(gpu):
     kvl = gu.i32_dev([1, 1])
     with pytest.raises(binding.VispecError):
         ctx.kv_compact(0, 1, gu.i32_dev(path), gu.i32_dev([2, 2]), kvl, kvl)                   # aliasing
+
+
+def _accept_commit_case(binding, gu, cfg_name, Hkv, D, layers, kv_len, S_max, seed=0):
+    """vispec_accept_commit against oracle.accept followed by oracle.kv_compact, whole buffers bit-exact."""
+    cfg = synth.get_config(cfg_name)
+    t = synth.make_tree_inputs(cfg)
+    B, N = cfg.B, cfg.N
+    rng = np.random.default_rng(seed)
+    ctx = binding.VerifyContext(B, N, Hkv, Hkv, D, S_max, layers)
+    host, dev = [], []
+    for l in range(layers):
+        k = rng.integers(0, 65536, size=(B, Hkv, S_max, D), dtype=np.int64).astype(np.uint16)
+        v = rng.integers(0, 65536, size=(B, Hkv, S_max, D), dtype=np.int64).astype(np.uint16)
+        kd, vd = gu.bf16_dev(k), gu.bf16_dev(v)
+        ctx.cache_register(l, kd, vd)
+        host.append((k, v)); dev.append((kd, vd))
+    path = torch.full((B, N), -9, dtype=torch.int32, device="cuda")
+    alen = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    bonus = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    out_len = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    ctx.accept_commit(0, layers, gu.i32_dev(t["draft_ids"]), gu.i32_dev(t["target_ids"]), gu.i32_dev(t["parents"]),
+                      gu.i32_dev(kv_len), path, alen, bonus, out_len)
+    torch.cuda.synchronize()
+    wp, wl, wb = oracle.accept(t["draft_ids"], t["target_ids"], t["parents"])
+    assert np.array_equal(path.cpu().numpy(), wp) and np.array_equal(alen.cpu().numpy(), wl)
+    assert np.array_equal(bonus.cpu().numpy(), wb)
+    for l in range(layers):
+        wk, wv, wn = oracle.kv_compact(host[l][0], host[l][1], wp, wl, kv_len)
+        assert np.array_equal(gu.bf16_bits(dev[l][0]), wk), f"K differs in layer {l}"
+        assert np.array_equal(gu.bf16_bits(dev[l][1]), wv), f"V differs in layer {l}"
+        assert np.array_equal(out_len.cpu().numpy(), wn)
+    assert ctx.status_poll() == 0
+    assert ctx.launch_count() == 1
+    return ctx
+
+
+def test_accept_commit_in_one_launch_matches_accept_then_compact(gpu):
+    binding, gu = gpu
+    _accept_commit_case(binding, gu, "llava13b_b4", 5, 128, 3, np.array([100, 37, 0, 250], dtype=np.int32), 320)
+    _accept_commit_case(binding, gu, "qwen3b_S2048_N128_B8", 2, 128, 2,
+                        np.array([0, 1, 127, 128, 129, 300, 77, 5], dtype=np.int32), 512, seed=3)
+    _accept_commit_case(binding, gu, "tiny", 4, 64, 1, np.array([256], dtype=np.int32), 320, seed=4)
+
+
+def test_accept_commit_bad_tree_and_overlong_sequence(gpu):
+    binding, gu = gpu
+    rng = np.random.default_rng(5)
+    B, Hkv, D, S_max, N = 2, 2, 64, 64, 4
+    ctx = binding.VerifyContext(B, N, Hkv, Hkv, D, S_max, 1)
+    k = rng.integers(0, 65536, size=(B, Hkv, S_max, D), dtype=np.int64).astype(np.uint16)
+    kd, vd = gu.bf16_dev(k), gu.bf16_dev(k)
+    ctx.cache_register(0, kd, vd)
+    path = torch.zeros((B, N), dtype=torch.int32, device="cuda")
+    alen = torch.zeros(B, dtype=torch.int32, device="cuda"); bonus = torch.zeros(B, dtype=torch.int32, device="cuda")
+    out_len = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    # sequence 0: invalid parent link -> root only; sequence 1: 61 + 4 > 64 -> accepted path reported, nothing committed
+    ctx.accept_commit(0, 1, gu.i32_dev([[0, 5, 6, 7], [0, 5, 6, 7]]), gu.i32_dev([[5, 6, 7, 8], [5, 6, 7, 8]]),
+                      gu.i32_dev([[-1, 0, 3, 1], [-1, 0, 1, 2]]), gu.i32_dev([10, 61]), path, alen, bonus, out_len)
+    torch.cuda.synchronize()
+    assert path.cpu().tolist() == [[0, -1, -1, -1], [0, 1, 2, 3]]
+    assert alen.cpu().tolist() == [1, 4] and bonus.cpu().tolist() == [5, 8]
+    assert out_len.cpu().tolist() == [11, -1]
+    assert np.array_equal(gu.bf16_bits(kd), k)            # root-only commit moves nothing; sequence 1 untouched
+    assert ctx.status_poll() in (-8, -4)                  # the first recorded of the two
