@@ -3,7 +3,7 @@
 
 A *step* is one pass of the whole hot path over one batch of synthetic input:
     vispec_tree_mask_build -> vispec_tree_verify_attn x L layers (each layer its own cache buffers)
-    -> vispec_accept -> vispec_kv_compact over all L layers.
+    -> vispec_accept_commit (acceptance + commit over all L layers in one launch).
 `value` is verify-attention KV GB/s: the K and V bytes the L attention calls must read
 (sum_b 2*(S_b+N)*Hkv*D*2 per layer) divided by the whole step's device time.  Inputs are resident in
 HBM before the timed region; the L layers' caches total far more than L2, so no flush is needed.
@@ -190,9 +190,9 @@ class DeviceWorkload:
             self.ctx.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
 
     def _post(self):
-        self.ctx.accept(self.draft, self.target, self.parents, self.path, self.alen, self.bonus)
-        # kv_len itself is left as it was so that every step sees the same workload
-        self.ctx.kv_compact(0, self.L, self.path, self.alen, self.kv_len, self.new_len)
+        # acceptance and commit in one launch; kv_len itself is left as it was so that every step sees the same workload
+        self.ctx.accept_commit(0, self.L, self.draft, self.target, self.parents, self.kv_len, self.path, self.alen,
+                               self.bonus, self.new_len)
 
     def capture(self):
         """Capture the three phases of a step as CUDA graphs (the launches are the same C-ABI calls;
@@ -275,8 +275,7 @@ class HostStep:
         c.tree_mask_build(parents, wl.mask, wl.depth)
         for l in range(wl.L):
             c.tree_verify_attn(l, wl.q[l], kv_len, wl.mask, wl.scale, wl.out[l])
-        c.accept(draft, target, parents, path, alen, bonus)
-        c.kv_compact(0, wl.L, path, alen, kv_len, new_len)
+        c.accept_commit(0, wl.L, draft, target, parents, kv_len, path, alen, bonus, new_len)
         self.h_out.copy_(wl.out, non_blocking=True)
         self.h_res.copy_(self.d_res, non_blocking=True)
         torch.cuda.current_stream().synchronize()      # the caller reads accept_len to go on
@@ -438,7 +437,7 @@ def main():
         "pct_of_8TBs": 100.0 * achieved / 8000.0,
         "status_word": status,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 3) // L} kernel launch(es) per call)",
+                     "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L} kernel launch(es) per call)",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)},
         "clocks": clocks,
         "gpu_launches": int(launches),

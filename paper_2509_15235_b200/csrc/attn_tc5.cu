@@ -277,10 +277,12 @@ __device__ unsigned long long g_timeline[4096][4];
 __device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 __device__ unsigned long long g_cta_times[256][4];
 #define CTA_T(k) do { if (threadIdx.x == 0 && blockIdx.x < 256) g_cta_times[blockIdx.x][k] = gtimer(); } while (0)
+#define CTA_TS(k) do { if (threadIdx.x == 128 && blockIdx.x < 256) g_cta_times[blockIdx.x][k] = gtimer(); } while (0)
 #define TL_START(idx, k) do { if ((idx) < 4096) atomicMin(&g_timeline[idx][k], gtimer()); } while (0)
 #define TL_END(idx, k) do { if ((idx) < 4096) atomicMax(&g_timeline[idx][k], gtimer()); } while (0)
 #else
 #define CTA_T(k) do {} while (0)
+#define CTA_TS(k) do {} while (0)
 #define TL_START(idx, k) do {} while (0)
 #define TL_END(idx, k) do {} while (0)
 #define TRACE(role, step, slot) do {} while (0)
@@ -581,6 +583,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         int px = 0;                                           // phases of the pair barrier used so far
         pdl_wait();                                           // q, tree_mask and every output come after the preceding kernel
         if (tid == 128) { TL_START(p.trace_idx, 2); TL_END(p.trace_idx, 3); }
+        CTA_TS(2);
         TRACE_MISC(4);
 
         // rejected sequences (kv_len < 0 or kv_len + N > S_max): zero output, -inf lse, status word
@@ -793,6 +796,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 // ---- segment epilogue: wait for the last product, add up the row statistics, (PAIR) merge the two
                 // halves, write out.  A thread owns columns [64 ch, 64 ch + 64) of its lane's accumulator row. ----
                 TRACE_MISC(5);
+                CTA_TS(3);
                 if (sg.n > 0) ok = mbar_wait_warp(bar(B_PVDONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
