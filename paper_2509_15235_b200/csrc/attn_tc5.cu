@@ -1140,7 +1140,8 @@ static int query_max_clusters(bool pair, int k) {
 }
 
 // Cluster size for the cluster form, or 0 when the even split with partials in global memory serves better:
-// one cluster per unit, all clusters co-resident, and most of the SMs in use.
+// one cluster per unit, all clusters co-resident, and at least three fifths of the SMs in use (one launch and no
+// partials in HBM outweigh the idle SMs down to about there).
 static int tc5_cluster_size(const AttnArgs& a, int units) {
     if (a.tc5_path == 1) return 0;
     const bool pair = (a.Hq / a.Hkv) * a.N <= 64;
@@ -1149,7 +1150,7 @@ static int tc5_cluster_size(const AttnArgs& a, int units) {
         if (units * k <= a.sm_count && g_max_clusters[pair][k] >= units) best = k;
     if (best == 0) return 0;
     if (a.tc5_path == 2) return best;
-    return (units * best * 4 >= a.sm_count * 3) ? best : 0;
+    return (units * best * 5 >= a.sm_count * 3) ? best : 0;
 }
 
 bool attn_tc5_supports(const AttnArgs& a) {
