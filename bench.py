@@ -189,6 +189,10 @@ class DeviceWorkload:
         for l in range(self.L):
             self.ctx.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
 
+    def _probe(self):
+        for l in range(self.L):
+            self.ctx.stream_probe(l, self.kv_len, self.cfg.N)
+
     def _post(self):
         # acceptance and commit in one launch; kv_len itself is left as it was so that every step sees the same workload
         self.ctx.accept_commit(0, self.L, self.draft, self.target, self.parents, self.kv_len, self.path, self.alen,
@@ -396,6 +400,29 @@ def main():
     kv_bytes_step = wl.kv_bytes_per_layer * L
     value = whole_job_gbs(kv_bytes_step, args.steps, ms_total * 1e-3, world)
 
+    # ---- streaming-read probe: the same K/V rows through the same TMA rings, no arithmetic (context for the roofline) ----
+    read_probe = None
+    if rank == 0 and cfg.D == 128 and cfg.B <= 32:
+        torch = wl.torch
+        g = torch.cuda.CUDAGraph()
+        wl._probe()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            wl._probe()
+        for _ in range(3):
+            g.replay()
+        n_probe = max(3, min(args.steps, 50))
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(n_probe):
+            g.replay()
+        r1.record()
+        torch.cuda.synchronize()
+        us = r0.elapsed_time(r1) * 1e3 / (n_probe * L)
+        read_probe = {"value": wl.kv_bytes_per_layer / (us * 1e-6) / 1e9, "unit": "GB/s", "us_per_layer": us,
+                      "what": "vispec_stream_probe: the K/V rows of one attention call through the same TMA rings, "
+                              "nothing computed, one launch per layer"}
+
     # ---- end-to-end timing (host buffers in, host results out) ----
     e2e = None
     if not args.no_e2e:
@@ -435,6 +462,7 @@ def main():
         "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
         "attn_us_per_layer": attn_s * 1e6,
         "pct_of_8TBs": 100.0 * achieved / 8000.0,
+        "read_probe": read_probe,
         "status_word": status,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L} kernel launch(es) per call)",

@@ -178,6 +178,14 @@ int vispec_tree_verify_attn_static(const void* q, const void* k_cache, const voi
                                    int Hq, int Hkv, int D, int S_max, float scale, void* out,
                                    float* lse, int* status_word, void* stream);
 
+/* Measurement aid (the paper has no counterpart): reads exactly the K and V rows that
+ * vispec_tree_verify_attn(layer, ..., kv_len, B, N) reads - slots [0, kv_len[b] + N) of every kv head, rounded
+ * up to whole 128-slot tiles - through the same TMA rings, on every SM, and does nothing with them.  Its time
+ * is the floor that streaming alone sets for an attention call on this machine.  D = 128 only (E_UNSUPPORTED
+ * otherwise), B <= 32.  Sequences with kv_len out of range are skipped.
+ * Host errors: E_NULL, E_SHAPE, E_RANGE (layer), E_UNREGISTERED, E_UNSUPPORTED. */
+int vispec_stream_probe(vispec_ctx* ctx, int layer, const int32_t* kv_len, int B, int N, void* stream);
+
 /* Greedy acceptance (Sec. 3.1 at temperature 0; Table 1 upper half).  target_ids[b][i] is the
  * target model's greedy token after node i; non-root node a is matched iff
  * draft_ids[b][a] == target_ids[b][parents[b][a]]; the accepted path ends at the deepest node whose

@@ -25,7 +25,7 @@ EXPORTS = [
     "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
     "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
-    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit",
+    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
@@ -68,6 +68,7 @@ def load() -> ctypes.CDLL:
             "vispec_accept": [vp, vp, vp, vp, ci, ci, vp, vp, vp, vp],
             "vispec_kv_compact": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp],
             "vispec_accept_commit": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp],
+            "vispec_stream_probe": [vp, ci, vp, ci, ci, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
             "vispec_tree_verify_attn_static": [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp],
@@ -193,6 +194,10 @@ class VerifyContext:
         _check(self.lib.vispec_accept_commit(self.handle, layer_begin, layer_end, _ptr(draft_ids), _ptr(target_ids),
                                              _ptr(parents), _ptr(kv_len), B, N, _ptr(path), _ptr(accept_len),
                                              _ptr(bonus), _ptr(kv_len_out), _stream()), "vispec_accept_commit")
+
+    def stream_probe(self, layer: int, kv_len: torch.Tensor, N: int) -> None:
+        _check(self.lib.vispec_stream_probe(self.handle, layer, _ptr(kv_len), kv_len.shape[0], N, _stream()),
+               "vispec_stream_probe")
 
     # -- diagnostics ------------------------------------------------------------------------------
     def status_poll(self) -> int:

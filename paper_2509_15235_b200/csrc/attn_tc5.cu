@@ -1122,6 +1122,81 @@ extern "C" int vispec_debug_timeline(unsigned long long* host, int reset) {
 
 static size_t tc5_partial_bytes(int grid, int rows) { return (size_t)2 * grid * rows * (D * 4 + 8); }
 
+namespace {
+
+// Streaming-read probe: the K/V rows one attention call reads, moved by the same TMA producer through the same
+// rings on the even split of all steps over the CTAs, and nothing else (a second thread hands every stage
+// straight back).  It measures what this way of streaming reaches on its own: the ceiling the attention kernel
+// can approach.
+__global__ void __launch_bounds__(64, 1)
+stream_probe_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const Tc5Params p) {
+    extern __shared__ __align__(1024) unsigned char sm[];
+    const uint32_t base = smem_u32(sm);
+    if (base & 1023u) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)VISPEC_E_UNSUPPORTED);
+        return;
+    }
+    constexpr int NS = NSK + NSV;                              // stages: K and V of a step take consecutive ones
+    const uint32_t bars = base + NS * STAGE_BYTES;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + NS * STAGE_BYTES + 2 * NS * 8);
+    Sched& sched = *reinterpret_cast<Sched*>(sm + NS * STAGE_BYTES + 256);
+    auto full = [&](int i) { return bars + 8u * (uint32_t)i; };
+    auto empty = [&](int i) { return bars + 8u * (uint32_t)(NS + i); };
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int i = 0; i < NS; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) sched_build(sched, p, lane);
+    pdl_launch_dependents();
+    if (!p.early) pdl_wait();
+    __syncthreads();
+    const int T = sched.base[p.B];
+    const int geff = T > 0 ? sched_ctas(T, sched.units, (int)gridDim.x, p.min_steps) : 0;
+    const int cta = blockIdx.x;
+    if (cta < geff && lane == 0) {
+        const int lo = cta_lo(cta, T, geff), hi = cta_lo(cta + 1, T, geff);
+        SegIter si; si.s = &sched; si.B = p.B; si.n_mblocks = p.n_mblocks; si.g = lo; si.lo = lo; si.hi = hi; si.cta = cta;
+        si.cl = false; si.cl_done = false;
+        Seg sg;
+        int n = 0;                                             // stages handled so far
+        if (warp == 0) {
+            const uint64_t pol = l2_evict_first_policy();
+            bool waited = !p.early, ok = true;
+            while (ok && si.next(sg)) {
+                const int bh = sg.b * p.Hkv + sg.kvh;
+                for (int t = 0; t < sg.n && ok; ++t) {
+                    const int tok = (sg.st0 + t) * STEP;
+                    if (!waited && tok + STEP > sg.S) { pdl_wait(); waited = true; }
+                    for (int kv = 0; kv < 2; ++kv, ++n) {
+                        const int s = n % NS;
+                        if (!mbar_wait(empty(s), ((n / NS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(full(s), STAGE_BYTES);
+                        tma_load_3d(base + s * STAGE_BYTES, kv ? &v_map : &k_map, full(s), 0, tok, bh, pol);
+                        tma_load_3d(base + s * STAGE_BYTES + HALF_BYTES, kv ? &v_map : &k_map, full(s), 64, tok, bh, pol);
+                    }
+                }
+            }
+            if (*abort_flag) {
+                volatile int never = 0;
+                for (int u = max(0, n - NS); u < n; ++u) mbar_wait(full(u % NS), (u / NS) & 1, &never);
+            }
+        } else {
+            bool ok = true;
+            while (ok && si.next(sg))
+                for (int t = 0; t < 2 * sg.n; ++t, ++n) {
+                    if (!mbar_wait(full(n % NS), (n / NS) & 1, abort_flag)) { ok = false; break; }
+                    mbar_arrive(empty(n % NS));
+                }
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && *abort_flag) atomicCAS(p.status, 0, (int)VISPEC_E_TIMEOUT);
+}
+
+}  // namespace
+
 // Largest number of co-resident clusters of each size (index: PAIR, cluster size), found once per device.
 static int g_max_clusters[2][9];
 
@@ -1225,6 +1300,27 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     if (err != cudaSuccess) return err;
     ++*n_launches;
     return cudaSuccess;
+}
+
+cudaError_t init_stream_probe() {
+    return cudaFuncSetAttribute(stream_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (NSK + NSV) * STAGE_BYTES + 256 + (int)sizeof(Sched));
+}
+
+cudaError_t launch_stream_probe(const AttnArgs& a, cudaStream_t st) {
+    const int rows_total = (a.Hq / a.Hkv) * a.N;
+    const int n_mblocks = rows_total <= 64 ? 1 : (rows_total + 127) / 128;
+    Tc5Params p = {};
+    p.kv_len = a.kv_len;
+    p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_max = a.S_max;
+    p.n_mblocks = 1;                                       // every K/V row once, whatever the number of row blocks
+    (void)n_mblocks;
+    const long long t_max = (long long)a.B * a.Hkv * ((a.S_max + STEP - 1) / STEP);
+    const int grid = (int)(t_max < a.sm_count ? t_max : a.sm_count);
+    p.grid_attn = grid; p.min_steps = 2; p.early = a.early_prefetch ? 1 : 0;
+    p.status = a.status;
+    return launch_pdl(stream_probe_kernel, dim3(grid), dim3(64), (size_t)((NSK + NSV) * STAGE_BYTES + 256 + sizeof(Sched)), st, 0,
+                      *a.k_map, *a.v_map, p);
 }
 
 }  // namespace vispec

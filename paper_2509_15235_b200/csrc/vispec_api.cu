@@ -83,6 +83,7 @@ int vispec_ctx_create(vispec_ctx** out, const vispec_shape* s, int device) {
     ok = ok && cudaMemset(c->d_cache_ptrs, 0, sizeof(void*) * 2 * s->layers) == cudaSuccess;
     ok = ok && init_attn_generic() == cudaSuccess;
     ok = ok && init_attn_tc5() == cudaSuccess;
+    ok = ok && init_stream_probe() == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { vispec_ctx_destroy(c); return VISPEC_E_CUDA; }
     c->h_k.assign(s->layers, nullptr);
@@ -199,6 +200,23 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
                                                                   : launch_attn_generic(a, (cudaStream_t)stream, &n);
     c->launches += n;
     return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
+}
+
+int vispec_stream_probe(vispec_ctx* c, int layer, const int32_t* kv_len, int B, int N, void* stream) {
+    if (!c || !kv_len) return VISPEC_E_NULL;
+    const vispec_shape& s = c->shape;
+    if (B < 1 || B > s.B_max || B > 32 || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
+    if (s.D != 128) return VISPEC_E_UNSUPPORTED;
+    if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
+    if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
+    AttnArgs a = {};
+    a.k = c->h_k[layer]; a.v = c->h_v[layer]; a.kv_len = kv_len;
+    a.B = B; a.N = N; a.Hq = s.Hq; a.Hkv = s.Hkv; a.D = s.D; a.S_max = s.S_max;
+    a.status = c->d_status; a.sm_count = c->sm_count; a.early_prefetch = c->early_prefetch;
+    a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
+    if (launch_stream_probe(a, (cudaStream_t)stream) != cudaSuccess) return VISPEC_E_CUDA;
+    c->launches += 1;
+    return VISPEC_OK;
 }
 
 int vispec_accept(vispec_ctx* c, const int32_t* draft_ids, const int32_t* target_ids, const int32_t* parents,

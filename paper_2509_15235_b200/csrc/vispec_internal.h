@@ -71,5 +71,8 @@ cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, int* n_launc
 bool attn_tc5_supports(const AttnArgs& a);
 cudaError_t init_attn_tc5();           // once per device, with that device current
 cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches);
+// Streaming-read probe over the rows one attention call reads (measurement aid).
+cudaError_t init_stream_probe();
+cudaError_t launch_stream_probe(const AttnArgs& a, cudaStream_t st);
 
 }  // namespace vispec

@@ -258,3 +258,24 @@ def test_redundant_image_keys_stress_the_softmax(gu):
         vis = list(range(S)) + [S + t for t in range(N) if (int(mask[0, i, 0]) >> t) & 1]
         for h in range(Hq):
             assert np.abs(out[0, i, h] - vf[0, h // (Hq // Hkv), vis].mean(axis=0)).max() <= TOL
+
+
+def test_stream_probe_runs_and_validates_its_arguments(gu):
+    """The measurement aid: it only reads, so the check is that it runs clean on ragged lengths (including a
+    rejected sequence, which it skips) and that the host-side validation answers."""
+    from paper_2509_15235_b200 import binding
+    ctx = binding.VerifyContext(3, 60, 4, 2, 128, 1024, 2)
+    k = torch.zeros((3, 2, 1024, 128), dtype=torch.bfloat16, device="cuda")
+    ctx.cache_register(0, k, k.clone())
+    ctx.stream_probe(0, gu.i32_dev([900, 0, 1000]), 60)        # 1000 + 60 > 1024: skipped
+    torch.cuda.synchronize()
+    assert ctx.status_poll() == 0
+    with pytest.raises(binding.VispecError) as e:
+        ctx.stream_probe(1, gu.i32_dev([1, 2, 3]), 60)
+    assert e.value.code == -9                                   # layer 1 has no registered cache
+    ctx64 = binding.VerifyContext(1, 8, 2, 2, 64, 128, 1)
+    c = torch.zeros((1, 2, 128, 64), dtype=torch.bfloat16, device="cuda")
+    ctx64.cache_register(0, c, c.clone())
+    with pytest.raises(binding.VispecError) as e:
+        ctx64.stream_probe(0, gu.i32_dev([10]), 8)
+    assert e.value.code == -5                                   # D = 64: no TMA maps
