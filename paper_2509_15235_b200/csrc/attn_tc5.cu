@@ -1215,8 +1215,7 @@ static int query_max_clusters(bool pair, int k) {
 }
 
 // Cluster size for the cluster form, or 0 when the even split with partials in global memory serves better:
-// one cluster per unit, all clusters co-resident, and at least three fifths of the SMs in use (one launch and no
-// partials in HBM outweigh the idle SMs down to about there).
+// one cluster per unit, all clusters co-resident, and three quarters of the SMs in use (three fifths for short calls).
 static int tc5_cluster_size(const AttnArgs& a, int units) {
     if (a.tc5_path == 1) return 0;
     const bool pair = (a.Hq / a.Hkv) * a.N <= 64;
@@ -1225,7 +1224,11 @@ static int tc5_cluster_size(const AttnArgs& a, int units) {
         if (units * k <= a.sm_count && g_max_clusters[pair][k] >= units) best = k;
     if (best == 0) return 0;
     if (a.tc5_path == 2) return best;
-    return (units * best * 5 >= a.sm_count * 3) ? best : 0;
+    if (units * best * 4 >= a.sm_count * 3) return best;
+    // Fewer CTAs than that pay off only for short calls, where the second launch and the partials of the even
+    // split weigh more than the idle SMs: at most 8 steps per CTA if every SM were used.
+    const long long t_max = (long long)units * ((a.S_max + STEP - 1) / STEP);
+    return (units * best * 5 >= a.sm_count * 3 && t_max <= 8ll * a.sm_count) ? best : 0;
 }
 
 bool attn_tc5_supports(const AttnArgs& a) {
