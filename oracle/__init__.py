@@ -35,7 +35,7 @@ def _load() -> ctypes.CDLL:
     if _lib is None:
         _lib = ctypes.CDLL(build())
         for name in ("oracle_tree_mask", "oracle_tree_attn", "oracle_accept", "oracle_kv_compact",
-                     "oracle_num_threads"):
+                     "oracle_num_threads", "oracle_rope_rows"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -109,3 +109,17 @@ def kv_compact(k_cache, v_cache, path, accept_len, kv_len):
     if rc != 0:
         raise ValueError(f"oracle_kv_compact rejected its arguments (code {rc})")
     return k, v, out_len
+
+
+def rope_rows(q, k_new, v_new, positions, kv_len, k_cache, v_cache, theta: float):
+    """Rotary embedding of the tree's q / k rows and placement of the k / v rows at slots kv_len + i.
+    Returns (q', k_cache', v_cache', skipped) as new arrays; the inputs are not modified."""
+    q = _c(q, np.uint16).copy(); k_new = _c(k_new, np.uint16); v_new = _c(v_new, np.uint16)
+    positions = _c(positions, np.int32); kv_len = _c(kv_len, np.int32)
+    kc = _c(k_cache, np.uint16).copy(); vc = _c(v_cache, np.uint16).copy()
+    B, N, Hq, D = q.shape
+    _, Hkv, S_max, _ = kc.shape
+    assert k_new.shape == (B, N, Hkv, D) and v_new.shape == k_new.shape and positions.shape == (B, N)
+    rc = _load().oracle_rope_rows(_p(q), _p(k_new), _p(v_new), _p(positions), _p(kv_len), _p(kc), _p(vc),
+                                  ctypes.c_double(theta), B, N, Hq, Hkv, D, S_max)
+    return q, kc, vc, rc

@@ -16,6 +16,9 @@
  *                       half): a drafted token survives iff it equals the target's greedy
  *                       token at its parent; the result is the longest surviving root path
  *   oracle_kv_compact   commit of the accepted rows into the pre-allocated cache (App. A)
+ *   oracle_rope_rows    rotary position embedding of the tree's q and k rows and their placement in the
+ *                       cache (Sec. 3.2: the target LLM is used unchanged; LLaVA and Qwen2.5-VL rotate q and
+ *                       k by position, in the half-split pairing: element j with element j + D/2)
  *
  * Layouts (row-major, C order):
  *   q, out            [B, N, Hq, D]
@@ -198,4 +201,69 @@ int oracle_kv_compact(uint16_t* k_cache, uint16_t* v_cache, const int32_t* path,
         if (kv_len_out) kv_len_out[b] = S + L;
     }
     return 0;
+}
+
+static uint16_t f64_to_bf16(double x) {
+    /* one rounding to nearest even of the fp64 value: the bf16 neighbours of x are exactly
+     * representable in fp64, so compare against their midpoint */
+    float f = (float)x;                       /* may double-round; corrected below */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7f800000u) == 0x7f800000u) return (uint16_t)(u >> 16);   /* inf / nan */
+    uint32_t lo = u & 0xffff0000u;            /* truncation toward zero */
+    float flo, fhi;
+    uint32_t hi = lo + 0x10000u;
+    memcpy(&flo, &lo, sizeof flo);
+    memcpy(&fhi, &hi, sizeof fhi);
+    double dlo = (double)flo, dhi = (double)fhi;
+    if (fabs(x) < fabs(dlo)) {                /* (float)x rounded away from x across a bf16 boundary */
+        hi = lo; lo = lo - 0x10000u;
+        memcpy(&flo, &lo, sizeof flo); memcpy(&fhi, &hi, sizeof fhi);
+        dlo = (double)flo; dhi = (double)fhi;
+    }
+    double mid = 0.5 * (dlo + dhi);
+    double ax = fabs(x), amid = fabs(mid);
+    if (ax < amid) return (uint16_t)(lo >> 16);
+    if (ax > amid) return (uint16_t)(hi >> 16);
+    return (uint16_t)(((lo >> 16) & 1u) ? (hi >> 16) : (lo >> 16));      /* tie: even mantissa */
+}
+
+/* Rotary embedding of the tree rows, then their placement in the cache (the step before the attention):
+ *   angle(b,i,j) = positions[b][i] * theta^(-2j/D),  j < D/2
+ *   x'[j] = x[j] cos - x[j+D/2] sin,   x'[j+D/2] = x[j+D/2] cos + x[j] sin        (q and k rows)
+ * q [B,N,Hq,D] is rotated in place; rotated k_new [B,N,Hkv,D] and v_new (unchanged) go to slots
+ * kv_len[b] + i of k_cache / v_cache [B,Hkv,S_max,D].  bf16 in, fp64 arithmetic, one rounding to bf16.
+ * A sequence with kv_len < 0 or kv_len + N > S_max is skipped.  Returns the number of skipped sequences. */
+int oracle_rope_rows(uint16_t* q, const uint16_t* k_new, const uint16_t* v_new, const int32_t* positions,
+                     const int32_t* kv_len, uint16_t* k_cache, uint16_t* v_cache, double theta,
+                     int B, int N, int Hq, int Hkv, int D, int S_max) {
+    int skipped = 0, half = D / 2;
+    for (int b = 0; b < B; ++b) {
+        int S = kv_len[b];
+        if (S < 0 || S + N > S_max) { ++skipped; continue; }
+        for (int i = 0; i < N; ++i) {
+            double pos = (double)positions[(size_t)b * N + i];
+            for (int j = 0; j < half; ++j) {
+                double ang = pos * pow(theta, -2.0 * (double)j / (double)D);
+                double c = cos(ang), sn = sin(ang);
+                for (int h = 0; h < Hq; ++h) {
+                    uint16_t* row = q + (((size_t)b * N + i) * Hq + h) * D;
+                    double a = bf16_to_f64(row[j]), bb = bf16_to_f64(row[j + half]);
+                    row[j] = f64_to_bf16(a * c - bb * sn);
+                    row[j + half] = f64_to_bf16(bb * c + a * sn);
+                }
+                for (int h = 0; h < Hkv; ++h) {
+                    const uint16_t* src = k_new + (((size_t)b * N + i) * Hkv + h) * D;
+                    uint16_t* dst = k_cache + (((size_t)b * Hkv + h) * S_max + S + i) * D;
+                    double a = bf16_to_f64(src[j]), bb = bf16_to_f64(src[j + half]);
+                    dst[j] = f64_to_bf16(a * c - bb * sn);
+                    dst[j + half] = f64_to_bf16(bb * c + a * sn);
+                }
+            }
+            for (int h = 0; h < Hkv; ++h)
+                memcpy(v_cache + (((size_t)b * Hkv + h) * S_max + S + i) * D,
+                       v_new + (((size_t)b * N + i) * Hkv + h) * D, (size_t)D * sizeof(uint16_t));
+        }
+    }
+    return skipped;
 }
