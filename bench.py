@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context: 0 automatic, 1 partials + merge kernel, 2 clusters")
+    ap.add_argument("--with-rope", action="store_true", help="also run vispec_rope_tree_rows before each layer's attention")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying graphs")
     return ap.parse_args()
 
@@ -181,12 +182,30 @@ class DeviceWorkload:
         self.new_len = torch.zeros(B, dtype=torch.int32, device=dev)
         self.scale = 1.0 / math.sqrt(D)
         self.kv_bytes_per_layer = cfg.kv_bytes_per_layer(tree["kv_len"])
+        self.with_rope = False
+
+    def enable_rope(self, tree, theta):
+        """Also rotate the tree rows and write them into the cache before each layer's attention (the step that
+        precedes it in a decoder layer).  The rows fed in are seeded noise; positions are kv_len + depth."""
+        torch, cfg = self.torch, self.cfg
+        g = torch.Generator(device=self.dev).manual_seed(1234)
+        shape = (self.L, cfg.B, cfg.N, cfg.Hkv, cfg.D)
+        self.k_new = torch.randn(shape, generator=g, device=self.dev, dtype=torch.float32).to(torch.bfloat16)
+        self.v_new = torch.randn(shape, generator=g, device=self.dev, dtype=torch.float32).to(torch.bfloat16)
+        self._pre()
+        torch.cuda.synchronize()
+        self.positions = (self.kv_len[:, None] + self.depth).to(torch.int32).contiguous()
+        self.theta = theta
+        self.with_rope = True
 
     def _pre(self):
         self.ctx.tree_mask_build(self.parents, self.mask, self.depth)
 
     def _attn(self):
         for l in range(self.L):
+            if self.with_rope:
+                self.ctx.rope_tree_rows(l, self.q[l], self.k_new[l], self.v_new[l], self.positions, self.kv_len,
+                                        self.theta)
             self.ctx.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
 
     def _probe(self):
@@ -361,6 +380,8 @@ def main():
         from paper_2509_15235_b200 import binding
         wl.ctx.ctx_set_option(binding.OPT_SPLIT_FORM, args.split_form)
     L = wl.L
+    if args.with_rope:
+        wl.enable_rope(tree, 1e6 if cfg.name.startswith("qwen") else 1e4)
 
     def barrier():
         if world > 1:
@@ -458,6 +479,7 @@ def main():
                    "kv_bytes_per_layer": wl.kv_bytes_per_layer,
                    "l2": f"inputs larger than L2: {L} layers x {wl.kv_bytes_per_layer / 1e6:.1f} MB rotate, no flush",
                    "launch": "plain C-ABI calls" if args.no_graph else "C-ABI calls captured once, replayed as 3 CUDA graphs per step",
+                   "rope_tree_rows": bool(args.with_rope),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
         "attn_us_per_layer": attn_s * 1e6,
@@ -465,7 +487,7 @@ def main():
         "read_probe": read_probe,
         "status_word": status,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L} kernel launch(es) per call)",
+                     "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L - int(args.with_rope)} kernel launch(es) per call)",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)},
         "clocks": clocks,
         "gpu_launches": int(launches),

@@ -178,6 +178,20 @@ int vispec_tree_verify_attn_static(const void* q, const void* k_cache, const voi
                                    int Hq, int Hkv, int D, int S_max, float scale, void* out,
                                    float* lse, int* status_word, void* stream);
 
+/* Rotary position embedding of the tree rows and their placement in the cache: the step just before
+ * vispec_tree_verify_attn of the same layer (Sec. 3.2: the target LLM runs unchanged; LLaVA-v1.6 and
+ * Qwen2.5-VL rotate q and k by position, pairing element j with element j + D/2).  For node i of sequence b
+ * and j < D/2:   angle = positions[b][i] * theta^(-2j/D)
+ *   x'[j] = x[j] cos(angle) - x[j+D/2] sin(angle),   x'[j+D/2] = x[j+D/2] cos(angle) + x[j] sin(angle)
+ * q [B,N,Hq,D] bf16 is rotated IN PLACE; k_new [B,N,Hkv,D] is rotated and written, v_new [B,N,Hkv,D] copied,
+ * to slots kv_len[b] + i of the caches registered for `layer`.  Angles and the rotation are formed in fp64,
+ * with one rounding to bf16.  positions is what the interface names (kv_len + depth for a draft tree); theta is
+ * the rotary base (> 1; 10000 for Vicuna, 1000000 for Qwen2.5).  A sequence with kv_len < 0 or kv_len + N > S_max
+ * is skipped with status word VISPEC_E_RANGE.
+ * Host errors: E_NULL, E_ALIGN (16 B), E_SHAPE, E_RANGE (layer), E_UNREGISTERED. */
+int vispec_rope_tree_rows(vispec_ctx* ctx, int layer, void* q, const void* k_new, const void* v_new,
+                          const int32_t* positions, const int32_t* kv_len, int B, int N, float theta, void* stream);
+
 /* Measurement aid (the paper has no counterpart): reads exactly the K and V rows that
  * vispec_tree_verify_attn(layer, ..., kv_len, B, N) reads - slots [0, kv_len[b] + N) of every kv head, rounded
  * up to whole 128-slot tiles - through the same TMA rings, on every SM, and does nothing with them.  Its time

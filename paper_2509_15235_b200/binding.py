@@ -25,7 +25,7 @@ EXPORTS = [
     "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
     "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
-    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe",
+    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
@@ -69,6 +69,7 @@ def load() -> ctypes.CDLL:
             "vispec_kv_compact": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp],
             "vispec_accept_commit": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp],
             "vispec_stream_probe": [vp, ci, vp, ci, ci, vp],
+            "vispec_rope_tree_rows": [vp, ci, vp, vp, vp, vp, vp, ci, ci, cf, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
             "vispec_tree_verify_attn_static": [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp],
@@ -194,6 +195,13 @@ class VerifyContext:
         _check(self.lib.vispec_accept_commit(self.handle, layer_begin, layer_end, _ptr(draft_ids), _ptr(target_ids),
                                              _ptr(parents), _ptr(kv_len), B, N, _ptr(path), _ptr(accept_len),
                                              _ptr(bonus), _ptr(kv_len_out), _stream()), "vispec_accept_commit")
+
+    def rope_tree_rows(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                       positions: torch.Tensor, kv_len: torch.Tensor, theta: float) -> None:
+        B, N = positions.shape
+        _check(self.lib.vispec_rope_tree_rows(self.handle, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(positions),
+                                              _ptr(kv_len), B, N, ctypes.c_float(theta), _stream()),
+               "vispec_rope_tree_rows")
 
     def stream_probe(self, layer: int, kv_len: torch.Tensor, N: int) -> None:
         _check(self.lib.vispec_stream_probe(self.handle, layer, _ptr(kv_len), kv_len.shape[0], N, _stream()),

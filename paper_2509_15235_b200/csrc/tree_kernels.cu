@@ -1,5 +1,7 @@
 // Integer kernels of the verification step: ancestor mask, greedy acceptance, KV commit.
 // All three are latency-bound (a few KB of traffic); each is a single launch.
+#include <cuda_bf16.h>
+
 #include "vispec_internal.h"
 
 namespace vispec {
@@ -269,6 +271,99 @@ cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int l
     accept_commit_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, draft, target, parents, kv_len, path,
                                                accept_len, bonus, kv_len_out, N, Hkv, D, S_max, status);
     return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rotary embedding of the tree's q and k rows and placement of the k and v rows at slots S + i (the step
+// before the attention; Sec. 3.2: the target LLM is unchanged, and LLaVA-v1.6 / Qwen2.5-VL rotate q and k by
+// position with the half-split pairing, element j with element j + D/2).  Each block forms the
+// D/2 angles positions[b][i] * theta^(-2j/D) of its (node, sequence) in fp64 (positions run into the thousands,
+// where fp32 argument reduction would cost digits), rotates its rows' pairs in fp64 and rounds once to bf16
+// (a few hundred thousand pairs: the arithmetic rate does not matter).  Latency-bound: about 1.5 MB per call.
+// ------------------------------------------------------------------------------------------------
+// Rows of one (node, sequence): Hq of q, Hkv of k, Hkv of v.  D/16 threads share a row, each holding 8 elements of
+// the lower half and the 8 they pair with in the upper half (two 16-byte loads, issued before any arithmetic); a
+// block covers 128 / (D/16) rows, blockIdx.z walks the rows, so the whole call is one wave of small blocks.
+__device__ __forceinline__ void rope_rotate8(uint4& lo, uint4& hi, const double* cs, const double* sn) {
+    __nv_bfloat16* a = reinterpret_cast<__nv_bfloat16*>(&lo);
+    __nv_bfloat16* b = reinterpret_cast<__nv_bfloat16*>(&hi);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const double x = (double)__bfloat162float(a[t]), y = (double)__bfloat162float(b[t]);
+        a[t] = __double2bfloat16(x * cs[t] - y * sn[t]);
+        b[t] = __double2bfloat16(y * cs[t] + x * sn[t]);
+    }
+}
+
+__global__ void __launch_bounds__(128)
+rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
+                 const __nv_bfloat16* __restrict__ v_new, const int32_t* __restrict__ positions,
+                 const int32_t* __restrict__ kv_len, __nv_bfloat16* __restrict__ k_cache,
+                 __nv_bfloat16* __restrict__ v_cache, double log2_theta, int N, int Hq, int Hkv, int D, int S_max,
+                 int* status) {
+    __shared__ double cs[64], sn[64];
+    // The attention that follows may start its prologue (and stream cache rows below kv_len, which this kernel never
+    // writes) while these blocks run; it waits for this grid to finish before it reads q or a tree row.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // q / k_new / v_new may come from the kernel just before
+    const int i = blockIdx.x, b = blockIdx.y, half = D / 2;
+    const int S = kv_len[b];
+    if (S < 0 || S + N > S_max) {
+        if (threadIdx.x == 0 && i == 0 && blockIdx.z == 0) record_status(status, VISPEC_E_RANGE);
+        return;
+    }
+    const int tpr = D / 16;                                   // threads per row
+    const int row = blockIdx.z * (128 / tpr) + threadIdx.x / tpr, c8 = (threadIdx.x % tpr) * 8;
+    const int rows = Hq + 2 * Hkv;
+    // this thread's two vectors: source and destination
+    const uint4* src = nullptr;
+    uint4* dst = nullptr;
+    if (row < Hq) {
+        __nv_bfloat16* r = q + (((size_t)b * N + i) * Hq + row) * D;
+        src = reinterpret_cast<const uint4*>(r);
+        dst = reinterpret_cast<uint4*>(r);
+    } else if (row < rows) {
+        const bool is_k = row < Hq + Hkv;
+        const int hk = row - Hq - (is_k ? 0 : Hkv);
+        src = reinterpret_cast<const uint4*>((is_k ? k_new : v_new) + (((size_t)b * N + i) * Hkv + hk) * D);
+        dst = reinterpret_cast<uint4*>((is_k ? k_cache : v_cache) + (((size_t)b * Hkv + hk) * S_max + S + i) * D);
+    }
+    uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
+    if (src) {
+        lo = src[c8 / 8];
+        hi = src[(c8 + half) / 8];
+    }
+    if ((int)threadIdx.x < half) {
+        const double ang = (double)positions[(size_t)b * N + i] * exp2(-2.0 * (double)threadIdx.x / (double)D * log2_theta);
+        double s_, c_;
+        sincos(ang, &s_, &c_);
+        cs[threadIdx.x] = c_;
+        sn[threadIdx.x] = s_;
+    }
+    __syncthreads();
+    if (!src) return;
+    if (row < Hq + Hkv) rope_rotate8(lo, hi, cs + c8, sn + c8);
+    dst[c8 / 8] = lo;
+    dst[(c8 + half) / 8] = hi;
+}
+
+cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,
+                             const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
+                             int Hkv, int D, int S_max, int* status, cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    const int rows_per_block = 128 / (D / 16);
+    cfg.gridDim = dim3(N, B, (Hq + 2 * Hkv + rows_per_block - 1) / rows_per_block);
+    cfg.blockDim = dim3(128);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, rope_rows_kernel, (__nv_bfloat16*)q, (const __nv_bfloat16*)k_new,
+                              (const __nv_bfloat16*)v_new, positions, kv_len, (__nv_bfloat16*)k_cache,
+                              (__nv_bfloat16*)v_cache, log2((double)theta), N, Hq, Hkv, D, S_max, status);
 }
 
 }  // namespace vispec

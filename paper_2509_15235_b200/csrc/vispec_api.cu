@@ -202,6 +202,21 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
     return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
 }
 
+int vispec_rope_tree_rows(vispec_ctx* c, int layer, void* q, const void* k_new, const void* v_new,
+                          const int32_t* positions, const int32_t* kv_len, int B, int N, float theta, void* stream) {
+    if (!c || !q || !k_new || !v_new || !positions || !kv_len) return VISPEC_E_NULL;
+    if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return VISPEC_E_ALIGN;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max || !(theta > 1.f)) return VISPEC_E_SHAPE;
+    if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
+    if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
+    if (launch_rope_rows(q, k_new, v_new, positions, kv_len, c->h_k[layer], c->h_v[layer], theta, B, N, s.Hq, s.Hkv,
+                         s.D, s.S_max, c->d_status, (cudaStream_t)stream) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
 int vispec_stream_probe(vispec_ctx* c, int layer, const int32_t* kv_len, int B, int N, void* stream) {
     if (!c || !kv_len) return VISPEC_E_NULL;
     const vispec_shape& s = c->shape;

@@ -50,6 +50,10 @@ cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int l
                                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, int B, int N,
                                  int Hkv, int D, int S_max, int* status, cudaStream_t st);
 
+cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,
+                             const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
+                             int Hkv, int D, int S_max, int* status, cudaStream_t st);
+
 struct AttnArgs {
     const void* q; const void* k; const void* v;
     const int32_t* kv_len; const uint64_t* mask;
