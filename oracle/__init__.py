@@ -35,7 +35,7 @@ def _load() -> ctypes.CDLL:
     if _lib is None:
         _lib = ctypes.CDLL(build())
         for name in ("oracle_tree_mask", "oracle_tree_attn", "oracle_accept", "oracle_kv_compact",
-                     "oracle_num_threads", "oracle_rope_rows"):
+                     "oracle_num_threads", "oracle_rope_rows", "oracle_accept_sampled"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -95,6 +95,25 @@ def accept(draft_ids, target_ids, parents):
     if rc != 0:
         raise ValueError(f"oracle_accept rejected its arguments (code {rc})")
     return path, alen, bonus
+
+
+def accept_sampled(draft_ids, parents, p, p_hat, u_accept, u_bonus):
+    """Sampled acceptance.  p, p_hat [B,N,V] float32; u_accept [B,N], u_bonus [B] float32 in [0,1).
+    -> (path [B,N] int32 padded with -1, accept_len [B], bonus [B], number of invalid sequences)."""
+    draft_ids = _c(draft_ids, np.int32); parents = _c(parents, np.int32)
+    p = _c(p, np.float32); p_hat = _c(p_hat, np.float32)
+    u_accept = _c(u_accept, np.float32); u_bonus = _c(u_bonus, np.float32)
+    B, N, V = p.shape
+    assert p_hat.shape == p.shape and parents.shape == (B, N) and draft_ids.shape == (B, N)
+    assert u_accept.shape == (B, N) and u_bonus.shape == (B,)
+    path = np.zeros((B, N), dtype=np.int32)
+    alen = np.zeros(B, dtype=np.int32)
+    bonus = np.zeros(B, dtype=np.int32)
+    rc = _load().oracle_accept_sampled(_p(draft_ids), _p(parents), _p(p), _p(p_hat), _p(u_accept), _p(u_bonus),
+                                       B, N, V, _p(path), _p(alen), _p(bonus))
+    if rc < 0:
+        raise MemoryError("oracle_accept_sampled")
+    return path, alen, bonus, rc
 
 
 def kv_compact(k_cache, v_cache, path, accept_len, kv_len):

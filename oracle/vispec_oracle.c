@@ -16,6 +16,11 @@
  *                       half): a drafted token survives iff it equals the target's greedy
  *                       token at its parent; the result is the longest surviving root path
  *   oracle_kv_compact   commit of the accepted rows into the pre-allocated cache (App. A)
+ *   oracle_accept_sampled  the acceptance rule of Sec. 3.1 at temperature > 0 (Table 1, lower half): a drafted
+ *                       token x is kept with probability min(1, p(x)/p^(x)); after a rejection the target
+ *                       distribution is replaced by norm(max(0, p - p^)); on a tree the rule is applied to
+ *                       the children of the current node one after the other (the tree of SpecInfer, which
+ *                       Sec. 3.1 cites), and the token after the last kept node is drawn from what remains
  *   oracle_rope_rows    rotary position embedding of the tree's q and k rows and their placement in the
  *                       cache (Sec. 3.2: the target LLM is used unchanged; LLaVA and Qwen2.5-VL rotate q and
  *                       k by position, in the half-split pairing: element j with element j + D/2)
@@ -169,6 +174,79 @@ int oracle_accept(const int32_t* draft_ids, const int32_t* target_ids, const int
         bonus[b] = tg[best];
     }
     return 0;
+}
+
+/* Draw from the unnormalised weights w[0..V) with one uniform u in [0,1): the smallest v whose running sum
+ * exceeds u * (sum of w); if rounding leaves none, the last v with w[v] > 0; -1 if no weight is positive. */
+static int32_t draw_from_weights(const double* w, int V, double u) {
+    double total = 0.0;
+    for (int v = 0; v < V; ++v) total += w[v];
+    if (!(total > 0.0)) return -1;
+    const double target = u * total;
+    double run = 0.0;
+    int32_t last = -1;
+    for (int v = 0; v < V; ++v) {
+        run += w[v];
+        if (w[v] > 0.0) last = v;
+        if (run > target) return v;
+    }
+    return last;
+}
+
+/* Sampled acceptance on a tree (Sec. 3.1, temperature > 0).
+ *   p      [B,N,V] fp32: row i = the target's distribution of the token that follows node i
+ *   p_hat  [B,N,V] fp32: row i = the draft distribution the tokens of node i's children were drawn from
+ *   draft_ids [B,N]: token of node i (the root's is the last sampled token and is always kept)
+ *   u_accept [B,N] in [0,1): the uniform that decides node i, if node i comes to be decided
+ *   u_bonus  [B]   in [0,1): the uniform that draws the token after the last kept node
+ * Walk: cur = root, r = p[cur].  The children of cur are decided in increasing index order: child c with token
+ * x is kept iff u_accept[c] < min(1, r[x] / p_hat[cur][x]) (0/0 counts as 0); if kept, cur = c, r = p[c], and the
+ * walk goes on with c's children; if not, r = norm(max(0, r - p_hat[cur])) and the next child is decided.  When
+ * cur has no child left, the bonus token is drawn from r.  If max(0, r - p_hat[cur]) is zero everywhere the walk
+ * stops and the bonus token is drawn from p[cur].
+ * path / accept_len / bonus as in oracle_accept.  A sequence whose parents are not earlier nodes, or with a
+ * drafted token outside [0,V), gets accept_len 0, path -1, bonus -1; the return value counts such sequences. */
+int oracle_accept_sampled(const int32_t* draft_ids, const int32_t* parents, const float* p, const float* p_hat,
+                          const float* u_accept, const float* u_bonus, int B, int N, int V,
+                          int32_t* path, int32_t* accept_len, int32_t* bonus) {
+    int bad = 0;
+    double* r = (double*)malloc(sizeof(double) * (size_t)V);
+    if (!r) return -1;
+    for (int b = 0; b < B; ++b) {
+        const int32_t* par = parents + (size_t)b * N;
+        const int32_t* dr = draft_ids + (size_t)b * N;
+        int32_t* pa = path + (size_t)b * N;
+        for (int k = 0; k < N; ++k) pa[k] = -1;
+        int ok = par[0] == -1;
+        for (int i = 1; i < N; ++i)
+            if (par[i] < 0 || par[i] >= i || dr[i] < 0 || dr[i] >= V) ok = 0;
+        if (!ok) { accept_len[b] = 0; bonus[b] = -1; ++bad; continue; }
+        int cur = 0, len = 1;
+        pa[0] = 0;
+        for (;;) {
+            const float* pt = p + ((size_t)b * N + cur) * V;
+            const float* ph = p_hat + ((size_t)b * N + cur) * V;
+            for (int v = 0; v < V; ++v) r[v] = (double)pt[v];
+            int kept = -1, empty = 0;
+            for (int c = cur + 1; c < N && kept < 0 && !empty; ++c) {
+                if (par[c] != cur) continue;
+                const int x = dr[c];
+                const double q = (double)ph[x];
+                const double ratio = q > 0.0 ? r[x] / q : (r[x] > 0.0 ? INFINITY : 0.0);
+                if ((double)u_accept[(size_t)b * N + c] < fmin(1.0, ratio)) { kept = c; break; }
+                double z = 0.0;
+                for (int v = 0; v < V; ++v) { r[v] = fmax(0.0, r[v] - (double)ph[v]); z += r[v]; }
+                if (z > 0.0) { for (int v = 0; v < V; ++v) r[v] /= z; }
+                else { empty = 1; for (int v = 0; v < V; ++v) r[v] = (double)pt[v]; }
+            }
+            if (kept >= 0) { cur = kept; pa[len++] = kept; continue; }
+            bonus[b] = draw_from_weights(r, V, (double)u_bonus[b]);
+            break;
+        }
+        accept_len[b] = len;
+    }
+    free(r);
+    return bad;
 }
 
 /* KV commit for one layer's cache pair: for every sequence and kv head the rows at slots
