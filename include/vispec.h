@@ -213,6 +213,27 @@ int vispec_accept(vispec_ctx* ctx, const int32_t* draft_ids, const int32_t* targ
                   const int32_t* parents, int B, int N, int32_t* path, int32_t* accept_len,
                   int32_t* bonus, void* stream);
 
+/* Sampled acceptance (Sec. 3.1 at temperature > 0; Table 1 lower half): a drafted token x is kept with
+ * probability min(1, p(x)/p^(x)); after a rejection the target distribution is replaced by
+ * norm(max(0, p - p^)).  On a tree the children of the current node are decided one after the other, in
+ * increasing node index (the multi-candidate form of the works Sec. 3.1 cites); the first kept child becomes the
+ * current node with its own target row; when no child is left the bonus token is drawn from what remains.
+ *   p_target [B,N,V] fp32 (device): row i = the target's distribution of the token after node i
+ *   p_draft  [B,N,V] fp32 (device): row i = the draft distribution node i's children were drawn from
+ *   u_accept [B,N] fp32 in [0,1): the uniform deciding node i (read only if node i comes to be decided)
+ *   u_bonus  [B]   fp32 in [0,1): draws the bonus token, as the smallest token whose running weight sum exceeds
+ *                  u_bonus * total (the last token of positive weight if rounding leaves none)
+ * The random numbers are inputs: the call is deterministic.  Decisions are taken in fp64 on the fp32 inputs.
+ * If max(0, r - p^) is zero everywhere after a rejection, the walk stops and the bonus token is drawn from the
+ * current node's target row; bonus = -1 if that row has no positive entry.
+ * path / accept_len / bonus as in vispec_accept (the outputs feed vispec_kv_compact unchanged).
+ * A sequence with invalid parents (status VISPEC_E_BAD_TREE) or a drafted token outside [0,V) (VISPEC_E_RANGE)
+ * gets accept_len 0, path -1, bonus -1.  draft_ids[b][0] is ignored.
+ * Host errors: E_NULL, E_ALIGN (rows 16 B), E_SHAPE. */
+int vispec_accept_sampled(vispec_ctx* ctx, const int32_t* draft_ids, const int32_t* parents, const float* p_target,
+                          const float* p_draft, const float* u_accept, const float* u_bonus, int B, int N, int V,
+                          int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream);
+
 /* Commit (App. A): for every registered layer in [layer_begin, layer_end), sequence and kv head, the
  * rows at slots S + path[b][k], k < accept_len[b], are gathered and then written to slots S + k, for
  * K and V, in place (gather-then-scatter: correct although a destination may be another entry's

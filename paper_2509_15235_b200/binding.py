@@ -25,7 +25,7 @@ EXPORTS = [
     "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
     "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
-    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows",
+    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows", "vispec_accept_sampled",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
@@ -69,6 +69,7 @@ def load() -> ctypes.CDLL:
             "vispec_kv_compact": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp],
             "vispec_accept_commit": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp],
             "vispec_stream_probe": [vp, ci, vp, ci, ci, vp],
+            "vispec_accept_sampled": [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp],
             "vispec_rope_tree_rows": [vp, ci, vp, vp, vp, vp, vp, ci, ci, cf, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
@@ -195,6 +196,14 @@ class VerifyContext:
         _check(self.lib.vispec_accept_commit(self.handle, layer_begin, layer_end, _ptr(draft_ids), _ptr(target_ids),
                                              _ptr(parents), _ptr(kv_len), B, N, _ptr(path), _ptr(accept_len),
                                              _ptr(bonus), _ptr(kv_len_out), _stream()), "vispec_accept_commit")
+
+    def accept_sampled(self, draft_ids: torch.Tensor, parents: torch.Tensor, p_target: torch.Tensor,
+                       p_draft: torch.Tensor, u_accept: torch.Tensor, u_bonus: torch.Tensor, path: torch.Tensor,
+                       accept_len: torch.Tensor, bonus: torch.Tensor) -> None:
+        B, N, V = p_target.shape
+        _check(self.lib.vispec_accept_sampled(self.handle, _ptr(draft_ids), _ptr(parents), _ptr(p_target), _ptr(p_draft),
+                                              _ptr(u_accept), _ptr(u_bonus), B, N, V, _ptr(path), _ptr(accept_len),
+                                              _ptr(bonus), _stream()), "vispec_accept_sampled")
 
     def rope_tree_rows(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
                        positions: torch.Tensor, kv_len: torch.Tensor, theta: float) -> None:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvispec.so")
-SOURCES = ["vispec_api.cu", "tree_kernels.cu", "attn_generic.cu", "attn_tc5.cu", "attn_static.cu"]
+SOURCES = ["vispec_api.cu", "tree_kernels.cu", "attn_generic.cu", "attn_tc5.cu", "attn_static.cu", "accept_sampled.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

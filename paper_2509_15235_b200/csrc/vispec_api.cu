@@ -245,6 +245,20 @@ int vispec_accept(vispec_ctx* c, const int32_t* draft_ids, const int32_t* target
     return VISPEC_OK;
 }
 
+int vispec_accept_sampled(vispec_ctx* c, const int32_t* draft_ids, const int32_t* parents, const float* p_target,
+                          const float* p_draft, const float* u_accept, const float* u_bonus, int B, int N, int V,
+                          int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
+    if (!c || !draft_ids || !parents || !p_target || !p_draft || !u_accept || !u_bonus || !path || !accept_len || !bonus)
+        return VISPEC_E_NULL;
+    if (!aligned(p_target, 16) || !aligned(p_draft, 16)) return VISPEC_E_ALIGN;
+    if (B < 0 || B > c->shape.B_max || N < 1 || N > c->shape.N_max || V < 1) return VISPEC_E_SHAPE;
+    if (launch_accept_sampled(draft_ids, parents, p_target, p_draft, u_accept, u_bonus, B, N, V, path, accept_len, bonus,
+                              c->d_status, (cudaStream_t)stream) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
 int vispec_kv_compact(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* path,
                       const int32_t* accept_len, const int32_t* kv_len, int32_t* kv_len_out, int B, int N,
                       void* stream) {

@@ -54,6 +54,10 @@ cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, cons
                              const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
                              int Hkv, int D, int S_max, int* status, cudaStream_t st);
 
+cudaError_t launch_accept_sampled(const int32_t* draft_ids, const int32_t* parents, const float* p, const float* p_hat,
+                                  const float* u_accept, const float* u_bonus, int B, int N, int V, int32_t* path,
+                                  int32_t* accept_len, int32_t* bonus, int* status, cudaStream_t st);
+
 struct AttnArgs {
     const void* q; const void* k; const void* v;
     const int32_t* kv_len; const uint64_t* mask;

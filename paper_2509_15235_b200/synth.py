@@ -194,6 +194,41 @@ def make_tree_inputs(cfg: VerifyConfig, seed_offset: int = 0) -> Dict[str, np.nd
     return {"parents": parents, "draft_ids": draft, "target_ids": target, "kv_len": kv_len}
 
 
+def softmax_rows_f32(logits: np.ndarray) -> np.ndarray:
+    """Row-wise softmax in float32 (an input recipe: what a model's head would hand over)."""
+    z = logits - logits.max(axis=-1, keepdims=True)
+    e = np.exp(z, dtype=np.float32)
+    return (e / e.sum(axis=-1, keepdims=True, dtype=np.float32)).astype(np.float32)
+
+
+def make_sampled_inputs(parents: np.ndarray, V: int, seed: int, sharpness: float = 6.0,
+                        disagreement: float = 0.3) -> Dict[str, np.ndarray]:
+    """Inputs of the sampled (temperature > 0) acceptance for given trees [B,N]:
+    p_target = softmax(sharpness * g), p_draft = softmax(sharpness * (g + disagreement * h)) with g, h i.i.d.
+    N(0,1) per (node, token): a few tokens carry most of the mass, the two models mostly agree; each non-root
+    node's token is drawn from its parent's draft row (i.i.d., so siblings may repeat); uniforms in [0,1)."""
+    B, N = parents.shape
+    rng = _rng(seed)
+    p = np.empty((B, N, V), dtype=np.float32)
+    ph = np.empty((B, N, V), dtype=np.float32)
+    for b in range(B):
+        g = rng.standard_normal((N, V), dtype=np.float32)
+        p[b] = softmax_rows_f32(np.float32(sharpness) * g)
+        g += np.float32(disagreement) * rng.standard_normal((N, V), dtype=np.float32)
+        ph[b] = softmax_rows_f32(np.float32(sharpness) * g)
+    ids = np.zeros((B, N), dtype=np.int32)
+    for b in range(B):
+        cdfs: Dict[int, np.ndarray] = {}
+        for i in range(1, N):
+            par = int(parents[b, i])
+            if par not in cdfs:
+                cdfs[par] = np.cumsum(ph[b, par].astype(np.float64))
+            cdf = cdfs[par]
+            ids[b, i] = min(int(np.searchsorted(cdf, rng.random() * cdf[-1], side="right")), V - 1)
+    return {"p_target": p, "p_draft": ph, "draft_ids": ids,
+            "u_accept": rng.random((B, N), dtype=np.float32), "u_bonus": rng.random(B, dtype=np.float32)}
+
+
 def make_layer_tensors(cfg: VerifyConfig, layer: int, S_max: Optional[int] = None,
                        seed_offset: int = 0) -> Dict[str, np.ndarray]:
     """One layer's bf16 tensors as uint16 bit patterns:
