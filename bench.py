@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context: 0 automatic, 1 partials + merge kernel, 2 clusters")
+    ap.add_argument("--no-sampled", action="store_true", help="skip the timing of vispec_accept_sampled")
     ap.add_argument("--with-rope", action="store_true", help="also run vispec_rope_tree_rows before each layer's attention")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying graphs")
     return ap.parse_args()
@@ -444,6 +445,38 @@ def main():
                       "what": "vispec_stream_probe: the K/V rows of one attention call through the same TMA rings, "
                               "nothing computed, one launch per layer"}
 
+    # ---- the step after the forward at temperature > 0: sampled acceptance on probability rows [B,N,V] ----
+    sampled = None
+    if rank == 0 and not args.no_sampled:
+        from paper_2509_15235_b200 import synth as _synth
+        si = _synth.make_sampled_inputs(tree["parents"], cfg.vocab, 777)
+        f32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(wl.dev)
+        # 8 input sets in rotation so that the probability rows come from HBM, not from L2
+        sets = [(f32(si["p_target"]), f32(si["p_draft"])) for _ in range(max(2, min(8, int(1.2e9 // si["p_target"].nbytes))))]
+        ids_d = torch.from_numpy(si["draft_ids"]).to(wl.dev)
+        ua_d, ub_d = f32(si["u_accept"]), f32(si["u_bonus"])
+        g = torch.cuda.CUDAGraph()
+        call = lambda pt, ph: wl.ctx.accept_sampled(ids_d, wl.parents, pt, ph, ua_d, ub_d, wl.path, wl.alen, wl.bonus)
+        call(*sets[0])
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            for pt, ph in sets:
+                call(pt, ph)
+        for _ in range(3):
+            g.replay()
+        n_rep = 20
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(n_rep):
+            g.replay()
+        r1.record()
+        torch.cuda.synchronize()
+        sampled = {"us_per_call": r0.elapsed_time(r1) * 1e3 / (n_rep * len(sets)), "vocab": cfg.vocab,
+                   "accept_len": [int(x) for x in wl.alen.cpu()],
+                   "what": "vispec_accept_sampled on synthetic probability rows [B,N,V] fp32, "
+                           f"{len(sets)} input sets in rotation, graph replay"}
+        assert wl.ctx.status_poll() == 0
+
     # ---- end-to-end timing (host buffers in, host results out) ----
     e2e = None
     if not args.no_e2e:
@@ -485,6 +518,7 @@ def main():
         "attn_us_per_layer": attn_s * 1e6,
         "pct_of_8TBs": 100.0 * achieved / 8000.0,
         "read_probe": read_probe,
+        "sampled_acceptance": sampled,
         "status_word": status,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L - int(args.with_rope)} kernel launch(es) per call)",

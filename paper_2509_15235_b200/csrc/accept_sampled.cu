@@ -10,7 +10,7 @@
 // bytes) to form the next S, and that pass also leaves per-warp partial sums that locate the bonus token, so the
 // draw re-reads one warp's slice only.
 //
-// One cluster per sequence (8 CTAs for large vocabularies, 1 for small ones), 512 threads per CTA.  Every CTA
+// One cluster per sequence (8 CTAs for large vocabularies, 1 for small ones), 1024 threads per CTA.  Every CTA
 // takes the same decisions from the same numbers: the CTA partials are exchanged through distributed shared
 // memory behind a hardware cluster barrier and summed by everyone in rank order, so S is bit-identical in the
 // cluster.  Sums and comparisons are fp64 (the inputs are fp32): the decisions then differ from a sequential
@@ -20,7 +20,7 @@
 namespace vispec {
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxCluster = 8;
 
@@ -71,7 +71,7 @@ __device__ __forceinline__ double slice_sum(const float* __restrict__ pt, const 
                                             Slice s, int lane) {
     double acc = 0.0;
     if (VEC) {
-#pragma unroll 4
+#pragma unroll 8
         for (int e = s.lo + lane * 4; e < s.hi; e += 128) {
             const float4 a = __ldg(reinterpret_cast<const float4*>(pt + e));
             const float4 b = __ldg(reinterpret_cast<const float4*>(ph + e));
@@ -110,6 +110,7 @@ accept_sampled_kernel(const int32_t* __restrict__ draft_ids, const int32_t* __re
                       int* status) {
     __shared__ int32_t par[VISPEC_MAX_TREE_NODES], ids[VISPEC_MAX_TREE_NODES], spath[VISPEC_MAX_TREE_NODES];
     __shared__ float ua[VISPEC_MAX_TREE_NODES];
+    __shared__ float px_of[VISPEC_MAX_TREE_NODES], phx_of[VISPEC_MAX_TREE_NODES];   // p[parent][token], p^[parent][token] per node
     __shared__ double seg[kWarps];               // this CTA's per-warp sums of the last pass
     __shared__ double part[2];                   // this CTA's sum, by pass parity (read by the whole cluster)
     __shared__ double allpart[kMaxCluster];      // every CTA's sum of the last pass
@@ -144,6 +145,14 @@ accept_sampled_kernel(const int32_t* __restrict__ draft_ids, const int32_t* __re
         return;
     }
 
+    // the two scalars each decision needs, for every node at once (one round of loads instead of one per decision)
+    if (tid >= 1 && tid < N) {
+        const size_t row = (nb + par[tid]) * (size_t)V + ids[tid];
+        px_of[tid] = __ldg(p + row);
+        phx_of[tid] = __ldg(p_hat + row);
+    }
+    __syncthreads();
+
     enum { PASS = 0, DRAW = 1 };
     // walk state, meaningful in thread 0 only
     int cur = 0, len = 1, next_child = 1;
@@ -153,8 +162,6 @@ accept_sampled_kernel(const int32_t* __restrict__ draft_ids, const int32_t* __re
 
     for (int iter = 0; iter < 2 * N + 4; ++iter) {
         if (tid == 0) {
-            const float* pt = p + (nb + cur) * (size_t)V;
-            const float* ph = p_hat + (nb + cur) * (size_t)V;
             int action = -1;
             while (action < 0) {
                 int ch = next_child;
@@ -163,16 +170,13 @@ accept_sampled_kernel(const int32_t* __restrict__ draft_ids, const int32_t* __re
                     action = have_pass ? DRAW : PASS;
                     break;
                 }
-                const int x = ids[ch];
-                const double px = (double)__ldg(pt + x), phx = (double)__ldg(ph + x);
+                const double px = (double)px_of[ch], phx = (double)phx_of[ch];
                 const double num = fmax(0.0, px - c * phx);
                 next_child = ch + 1;
                 if ((double)ua[ch] * S * phx < num) {          // kept: u < min(1, r(x)/p^(x)), r = m/S
                     cur = ch;
                     spath[len++] = ch;
                     c = 0.0; S = 1.0; have_pass = false;
-                    pt = p + (nb + cur) * (size_t)V;
-                    ph = p_hat + (nb + cur) * (size_t)V;
                 } else {                                        // rejected: next residual needs its sum
                     c += S;
                     action = PASS;
@@ -191,17 +195,24 @@ accept_sampled_kernel(const int32_t* __restrict__ draft_ids, const int32_t* __re
         __syncthreads();
         const int parity = iter & 1;
         if (tid == 0) {
+            double v[kWarps];
+#pragma unroll
+            for (int i = 0; i < kWarps; ++i) v[i] = seg[i];          // all loads first, then the ordered sum
             double t = 0.0;
-            for (int i = 0; i < kWarps; ++i) t += seg[i];
+#pragma unroll
+            for (int i = 0; i < kWarps; ++i) t += v[i];
             part[parity] = t;
         }
         cl_sync();                               // every CTA's part[parity] is written and visible
         if (tid == 0) {
+            double v[kMaxCluster];
+#pragma unroll
+            for (int r = 0; r < kMaxCluster; ++r) v[r] = r < csize ? cl_ld_f64(&part[parity], (uint32_t)r) : 0.0;
             double t = 0.0;
-            for (int r = 0; r < csize; ++r) {
-                const double v = cl_ld_f64(&part[parity], (uint32_t)r);
-                allpart[r] = v;
-                t += v;
+#pragma unroll
+            for (int r = 0; r < kMaxCluster; ++r) {
+                allpart[r] = v[r];
+                t += v[r];
             }
             if (t > 0.0) {
                 S = t; have_pass = true;
