@@ -35,7 +35,7 @@ def _load() -> ctypes.CDLL:
     if _lib is None:
         _lib = ctypes.CDLL(build())
         for name in ("oracle_tree_mask", "oracle_tree_attn", "oracle_accept", "oracle_kv_compact",
-                     "oracle_num_threads", "oracle_rope_rows", "oracle_accept_sampled"):
+                     "oracle_num_threads", "oracle_rope_rows", "oracle_accept_sampled", "oracle_tree_rerank"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -114,6 +114,22 @@ def accept_sampled(draft_ids, parents, p, p_hat, u_accept, u_bonus):
     if rc < 0:
         raise MemoryError("oracle_accept_sampled")
     return path, alen, bonus, rc
+
+
+def tree_rerank(cand_parent, cand_token, cand_score, K: int):
+    """Candidates [B,M] -> (parents [B,K+1], draft_ids [B,K+1], selected [B,K], number of invalid sequences)."""
+    cand_parent = _c(cand_parent, np.int32); cand_token = _c(cand_token, np.int32)
+    cand_score = _c(cand_score, np.float32)
+    B, M = cand_parent.shape
+    assert cand_token.shape == (B, M) and cand_score.shape == (B, M)
+    parents = np.zeros((B, K + 1), dtype=np.int32)
+    ids = np.zeros((B, K + 1), dtype=np.int32)
+    sel = np.zeros((B, K), dtype=np.int32)
+    rc = _load().oracle_tree_rerank(_p(cand_parent), _p(cand_token), _p(cand_score), B, M, K, _p(parents), _p(ids),
+                                    _p(sel))
+    if rc < 0:
+        raise ValueError(f"oracle_tree_rerank rejected its arguments (code {rc})")
+    return parents, ids, sel, rc
 
 
 def kv_compact(k_cache, v_cache, path, accept_len, kv_len):

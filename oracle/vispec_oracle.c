@@ -21,6 +21,9 @@
  *                       distribution is replaced by norm(max(0, p - p^)); on a tree the rule is applied to
  *                       the children of the current node one after the other (the tree of SpecInfer, which
  *                       Sec. 3.1 cites), and the token after the last kept node is drawn from what remains
+ *   oracle_tree_rerank  choice of the draft tree's nodes among the expansion's candidates (App. A: 30 draft
+ *                       tokens, depth 3, 8 nodes expanded per level; the tree is EAGLE-2's, which keeps the
+ *                       candidates of highest cumulative log-probability)
  *   oracle_rope_rows    rotary position embedding of the tree's q and k rows and their placement in the
  *                       cache (Sec. 3.2: the target LLM is used unchanged; LLaVA and Qwen2.5-VL rotate q and
  *                       k by position, in the half-split pairing: element j with element j + D/2)
@@ -246,6 +249,65 @@ int oracle_accept_sampled(const int32_t* draft_ids, const int32_t* parents, cons
         accept_len[b] = len;
     }
     free(r);
+    return bad;
+}
+
+/* a ranks before b: higher score first, NaN below everything, equal scores by lower index */
+static int ranks_before(const float* score, int a, int b) {
+    const float sa = score[a], sb = score[b];
+    const int na = isnan(sa), nb = isnan(sb);
+    if (na || nb) return na != nb ? nb : a < b;
+    if (sa != sb) return sa > sb;
+    return a < b;
+}
+
+/* Tree rerank: of M candidates (cand_parent[i] = an earlier candidate or -1 for a child of the root,
+ * cand_score[i] = cumulative log-probability of the path to i, cand_token[i]) keep the K of highest score
+ * (equal scores: lower index first; NaN last) and emit them in increasing candidate index as nodes 1..K of a
+ * tree whose node 0 is the root:
+ *   selected[b][j-1] = candidate index of node j;  parents[b][j] = node number of its parent (0 for -1);
+ *   draft_ids[b][j] = its token;  parents[b][0] = -1, draft_ids[b][0] = 0.
+ * A sequence with a parent index that is not an earlier candidate, or with a kept candidate whose parent
+ * was not kept, is counted in the return value and gets parents = -1 throughout (selected and draft_ids are
+ * still written). */
+int oracle_tree_rerank(const int32_t* cand_parent, const int32_t* cand_token, const float* cand_score,
+                       int B, int M, int K, int32_t* parents, int32_t* draft_ids, int32_t* selected) {
+    if (K < 0 || K > M) return -1;
+    int bad = 0;
+    int* keep = (int*)malloc(sizeof(int) * (size_t)(M > 0 ? M : 1));
+    int* node = (int*)malloc(sizeof(int) * (size_t)(M > 0 ? M : 1));
+    if (!keep || !node) { free(keep); free(node); return -2; }
+    for (int b = 0; b < B; ++b) {
+        const int32_t* cp = cand_parent + (size_t)b * M;
+        const int32_t* ct = cand_token + (size_t)b * M;
+        const float* cs = cand_score + (size_t)b * M;
+        int32_t* po = parents + (size_t)b * (K + 1);
+        int32_t* io = draft_ids + (size_t)b * (K + 1);
+        int32_t* so = selected + (size_t)b * K;
+        int ok = 1;
+        for (int i = 0; i < M; ++i) {
+            if (cp[i] < -1 || cp[i] >= i) ok = 0;
+            int ahead = 0;                                  /* how many candidates rank before i */
+            for (int j = 0; j < M; ++j)
+                if (j != i && ranks_before(cs, j, i)) ++ahead;
+            keep[i] = ahead < K;
+        }
+        po[0] = -1; io[0] = 0;
+        int n = 0;
+        for (int i = 0; i < M; ++i) {
+            node[i] = -1;
+            if (!keep[i]) continue;
+            node[i] = ++n;
+            so[n - 1] = i;
+            io[n] = ct[i];
+            if (!ok) continue;
+            if (cp[i] == -1) po[n] = 0;
+            else if (keep[cp[i]]) po[n] = node[cp[i]];
+            else ok = 0;
+        }
+        if (!ok) { ++bad; for (int j = 0; j <= K; ++j) po[j] = -1; }
+    }
+    free(keep); free(node);
     return bad;
 }
 

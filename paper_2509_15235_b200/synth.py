@@ -229,6 +229,41 @@ def make_sampled_inputs(parents: np.ndarray, V: int, seed: int, sharpness: float
             "u_accept": rng.random((B, N), dtype=np.float32), "u_bonus": rng.random(B, dtype=np.float32)}
 
 
+def make_rerank_candidates(B: int, depth: int, width: int, vocab: int, seed: int) -> Dict[str, np.ndarray]:
+    """Candidates of a level-by-level tree expansion (the input of the rerank): level 1 holds `width` children
+    of the root, every later level `width` children of each of the `width` best candidates of the level before
+    (best by cumulative score), so M = width + (depth - 1) * width^2 (136 for depth 3, width 8).  A child's score
+    is its parent's plus the log of one of the `width` largest entries of a random distribution over the
+    vocabulary (softmax of 3 * N(0,1)); its token is that entry's index."""
+    rng = _rng(seed)
+    M = width + (depth - 1) * width * width
+    parent = np.full((B, M), -1, dtype=np.int32)
+    token = np.zeros((B, M), dtype=np.int32)
+    score = np.zeros((B, M), dtype=np.float32)
+
+    def expand():
+        pr = softmax_rows_f32(np.float32(3.0) * rng.standard_normal((1, vocab), dtype=np.float32))[0]
+        top = np.argsort(-pr, kind="stable")[:width]
+        return top.astype(np.int32), np.log(pr[top]).astype(np.float32)
+
+    for b in range(B):
+        tok, lp = expand()
+        token[b, :width], score[b, :width] = tok, lp
+        level = list(range(width))
+        n = width
+        for _ in range(1, depth):
+            best = sorted(level, key=lambda i: (-float(score[b, i]), i))[:width]
+            level = []
+            for par in sorted(best):
+                tok, lp = expand()
+                token[b, n:n + width] = tok
+                score[b, n:n + width] = score[b, par] + lp
+                parent[b, n:n + width] = par
+                level.extend(range(n, n + width))
+                n += width
+    return {"cand_parent": parent, "cand_token": token, "cand_score": score}
+
+
 def make_layer_tensors(cfg: VerifyConfig, layer: int, S_max: Optional[int] = None,
                        seed_offset: int = 0) -> Dict[str, np.ndarray]:
     """One layer's bf16 tensors as uint16 bit patterns:
