@@ -476,6 +476,31 @@ def main():
                    "what": "vispec_accept_sampled on synthetic probability rows [B,N,V] fp32, "
                            f"{len(sets)} input sets in rotation, graph replay"}
         assert wl.ctx.status_poll() == 0
+        # the step before the forward: rerank of a depth-3, width-8 expansion down to N - 1 draft tokens
+        K = min(cfg.N - 1, 127)
+        width = 8
+        rdepth = max(3, -(-(K - width) // (width * width)) + 1)
+        rc = _synth.make_rerank_candidates(cfg.B, rdepth, width, cfg.vocab, 778)
+        cp_d, ct_d = (torch.from_numpy(rc[k]).to(wl.dev) for k in ("cand_parent", "cand_token"))
+        cs_d = f32(rc["cand_score"])
+        rp = torch.zeros((cfg.B, K + 1), dtype=torch.int32, device=wl.dev)
+        ri = torch.zeros_like(rp)
+        rs = torch.zeros((cfg.B, K), dtype=torch.int32, device=wl.dev)
+        g2 = torch.cuda.CUDAGraph()
+        wl.ctx.tree_rerank(cp_d, ct_d, cs_d, K, rp, ri, rs)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g2):
+            for _ in range(8):
+                wl.ctx.tree_rerank(cp_d, ct_d, cs_d, K, rp, ri, rs)
+        g2.replay()
+        r0.record()
+        for _ in range(n_rep):
+            g2.replay()
+        r1.record()
+        torch.cuda.synchronize()
+        sampled["tree_rerank_us_per_call"] = r0.elapsed_time(r1) * 1e3 / (n_rep * 8)
+        sampled["tree_rerank_candidates"] = int(cp_d.shape[1])
+        assert wl.ctx.status_poll() == 0
 
     # ---- end-to-end timing (host buffers in, host results out) ----
     e2e = None
@@ -518,7 +543,7 @@ def main():
         "attn_us_per_layer": attn_s * 1e6,
         "pct_of_8TBs": 100.0 * achieved / 8000.0,
         "read_probe": read_probe,
-        "sampled_acceptance": sampled,
+        "around_the_forward": sampled,
         "status_word": status,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L - int(args.with_rope)} kernel launch(es) per call)",

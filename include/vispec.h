@@ -200,6 +200,24 @@ int vispec_rope_tree_rows(vispec_ctx* ctx, int layer, void* q, const void* k_new
  * Host errors: E_NULL, E_SHAPE, E_RANGE (layer), E_UNREGISTERED, E_UNSUPPORTED. */
 int vispec_stream_probe(vispec_ctx* ctx, int layer, const int32_t* kv_len, int B, int N, void* stream);
 
+/* Tree rerank: the last step of building the draft tree, the one that needs scores only (App. A: 30 draft
+ * tokens kept from a depth-3 expansion of 8 nodes per level; the tree is EAGLE-2's, which keeps the candidates
+ * of highest cumulative log-probability).  Of M candidates per sequence
+ *   cand_parent [B,M] int32: an earlier candidate, or -1 for a child of the root
+ *   cand_token  [B,M] int32,  cand_score [B,M] fp32 (cumulative log-probability of the path to the candidate)
+ * the K of highest score are kept (equal scores: lower index first; NaN below everything) and become nodes
+ * 1..K of a tree in increasing candidate index (parents stay ahead of children); node 0 is the root:
+ *   parents   [B,K+1]: parents[b][0] = -1, parents[b][j] = node number of node j's parent
+ *   draft_ids [B,K+1]: draft_ids[b][0] = 0 (ignored downstream), draft_ids[b][j] = token of node j
+ *   selected  [B,K]:   candidate index of node j at [j-1] (may be NULL if K == 0)
+ * The outputs are the inputs of vispec_tree_mask_build / vispec_accept* with N = K + 1.  A sequence with a parent
+ * index that is not an earlier candidate, or a kept candidate whose parent was not kept (impossible for
+ * cumulative log-probabilities), gets parents = -1 throughout and the status word VISPEC_E_BAD_TREE; selected
+ * and draft_ids are still written.  Bit-exact: only comparisons of the given floats.
+ * Host errors: E_NULL, E_SHAPE (M in [1, 2048], 0 <= K <= M, K + 1 <= N_max). */
+int vispec_tree_rerank(vispec_ctx* ctx, const int32_t* cand_parent, const int32_t* cand_token, const float* cand_score,
+                       int B, int M, int K, int32_t* parents, int32_t* draft_ids, int32_t* selected, void* stream);
+
 /* Greedy acceptance (Sec. 3.1 at temperature 0; Table 1 upper half).  target_ids[b][i] is the
  * target model's greedy token after node i; non-root node a is matched iff
  * draft_ids[b][a] == target_ids[b][parents[b][a]]; the accepted path ends at the deepest node whose

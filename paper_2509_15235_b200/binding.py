@@ -25,7 +25,7 @@ EXPORTS = [
     "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
     "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
-    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows", "vispec_accept_sampled",
+    "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows", "vispec_accept_sampled", "vispec_tree_rerank",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
@@ -70,6 +70,7 @@ def load() -> ctypes.CDLL:
             "vispec_accept_commit": [vp, ci, ci, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp],
             "vispec_stream_probe": [vp, ci, vp, ci, ci, vp],
             "vispec_accept_sampled": [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp],
+            "vispec_tree_rerank": [vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp],
             "vispec_rope_tree_rows": [vp, ci, vp, vp, vp, vp, vp, ci, ci, cf, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
@@ -204,6 +205,13 @@ class VerifyContext:
         _check(self.lib.vispec_accept_sampled(self.handle, _ptr(draft_ids), _ptr(parents), _ptr(p_target), _ptr(p_draft),
                                               _ptr(u_accept), _ptr(u_bonus), B, N, V, _ptr(path), _ptr(accept_len),
                                               _ptr(bonus), _stream()), "vispec_accept_sampled")
+
+    def tree_rerank(self, cand_parent: torch.Tensor, cand_token: torch.Tensor, cand_score: torch.Tensor, K: int,
+                    parents: torch.Tensor, draft_ids: torch.Tensor, selected: Optional[torch.Tensor]) -> None:
+        B, M = cand_parent.shape
+        _check(self.lib.vispec_tree_rerank(self.handle, _ptr(cand_parent), _ptr(cand_token), _ptr(cand_score), B, M, K,
+                                           _ptr(parents), _ptr(draft_ids), _ptr(selected), _stream()),
+               "vispec_tree_rerank")
 
     def rope_tree_rows(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
                        positions: torch.Tensor, kv_len: torch.Tensor, theta: float) -> None:

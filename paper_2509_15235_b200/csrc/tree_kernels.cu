@@ -366,4 +366,95 @@ cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, cons
                               (__nv_bfloat16*)v_cache, log2((double)theta), N, Hq, Hkv, D, S_max, status);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Tree rerank (App. A: 30 draft tokens kept from a depth-3, width-8 expansion; the tree is EAGLE-2's, which
+// keeps the candidates of highest cumulative log-probability).  One block per sequence.  Scores become
+// order-preserving 32-bit keys (NaN lowest); a candidate's rank is the number of candidates ahead of it
+// (higher key, or equal key and lower index), counted against the keys in shared memory: M^2 compares,
+// 18 K for the paper's 136 candidates.  Kept candidates are numbered in candidate order, which keeps
+// parents ahead of children.
+// ------------------------------------------------------------------------------------------------
+constexpr int kRerankMaxM = 2048;
+
+__global__ void __launch_bounds__(256)
+tree_rerank_kernel(const int32_t* __restrict__ cand_parent, const int32_t* __restrict__ cand_token,
+                   const float* __restrict__ cand_score, int M, int K, int32_t* __restrict__ parents,
+                   int32_t* __restrict__ draft_ids, int32_t* __restrict__ selected, int* status) {
+    __shared__ uint32_t key[kRerankMaxM];
+    __shared__ int16_t node[kRerankMaxM];        // node number of a kept candidate, 0 if dropped
+    __shared__ int warp_cnt[8];
+    __shared__ int sh_bad;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int32_t* cp = cand_parent + (size_t)b * M;
+    if (tid == 0) sh_bad = 0;
+    for (int i = tid; i < M; i += 256) {
+        const float s = cand_score[(size_t)b * M + i];
+        const uint32_t u = __float_as_uint(s);
+        // ascending float order -> ascending unsigned order; -0 and +0 made equal; NaN below everything
+        uint32_t k = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+        if (s == 0.0f) k = 0x80000000u;
+        if (s != s) k = 0u;
+        key[i] = k;
+    }
+    __syncthreads();
+    // pass over the candidates in chunks of 256 (in index order) so that the node numbers can be handed out
+    // by a block-wide prefix count
+    int base = 0;
+    for (int i0 = 0; i0 < M; i0 += 256) {
+        const int i = i0 + tid;
+        bool keep = false;
+        if (i < M) {
+            const uint32_t ki = key[i];
+            int ahead = 0;
+            for (int j = 0; j < M; ++j) {
+                const uint32_t kj = key[j];
+                ahead += (kj > ki) || (kj == ki && j < i);
+            }
+            keep = ahead < K;
+            const int pr = cp[i];
+            if (pr < -1 || pr >= i) sh_bad = 1;
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) warp_cnt[w] = __popc(m);
+        __syncthreads();
+        int before = base + __popc(m & ((1u << lane) - 1));
+        for (int x = 0; x < w; ++x) before += warp_cnt[x];
+        int total = 0;
+        for (int x = 0; x < 8; ++x) total += warp_cnt[x];
+        if (i < M) node[i] = keep ? (int16_t)(before + 1) : (int16_t)0;
+        base += total;
+        __syncthreads();
+    }
+    // a kept candidate whose parent was dropped breaks the tree
+    for (int i = tid; i < M; i += 256) {
+        const int pr = cp[i];
+        if (node[i] && pr >= 0 && pr < i && !node[pr]) sh_bad = 1;
+    }
+    __syncthreads();
+    const bool bad = sh_bad != 0;
+    int32_t* po = parents + (size_t)b * (K + 1);
+    int32_t* io = draft_ids + (size_t)b * (K + 1);
+    if (tid == 0) {
+        po[0] = -1;
+        io[0] = 0;
+        if (bad) record_status(status, VISPEC_E_BAD_TREE);
+    }
+    for (int i = tid; i < M; i += 256) {
+        const int n = node[i];
+        if (!n) continue;
+        selected[(size_t)b * K + n - 1] = i;
+        io[n] = cand_token[(size_t)b * M + i];
+        const int pr = cp[i];
+        po[n] = bad ? -1 : (pr == -1 ? 0 : (int)node[pr]);
+    }
+}
+
+cudaError_t launch_tree_rerank(const int32_t* cand_parent, const int32_t* cand_token, const float* cand_score, int B,
+                               int M, int K, int32_t* parents, int32_t* draft_ids, int32_t* selected, int* status,
+                               cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    tree_rerank_kernel<<<B, 256, 0, st>>>(cand_parent, cand_token, cand_score, M, K, parents, draft_ids, selected, status);
+    return cudaGetLastError();
+}
+
 }  // namespace vispec

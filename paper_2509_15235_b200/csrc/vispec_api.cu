@@ -245,6 +245,19 @@ int vispec_accept(vispec_ctx* c, const int32_t* draft_ids, const int32_t* target
     return VISPEC_OK;
 }
 
+int vispec_tree_rerank(vispec_ctx* c, const int32_t* cand_parent, const int32_t* cand_token, const float* cand_score,
+                       int B, int M, int K, int32_t* parents, int32_t* draft_ids, int32_t* selected, void* stream) {
+    if (!c || !cand_parent || !cand_token || !cand_score || !parents || !draft_ids || (!selected && K > 0))
+        return VISPEC_E_NULL;
+    if (B < 0 || B > c->shape.B_max || M < 1 || M > 2048 || K < 0 || K > M || K + 1 > c->shape.N_max)
+        return VISPEC_E_SHAPE;
+    if (launch_tree_rerank(cand_parent, cand_token, cand_score, B, M, K, parents, draft_ids, selected, c->d_status,
+                           (cudaStream_t)stream) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
 int vispec_accept_sampled(vispec_ctx* c, const int32_t* draft_ids, const int32_t* parents, const float* p_target,
                           const float* p_draft, const float* u_accept, const float* u_bonus, int B, int N, int V,
                           int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {

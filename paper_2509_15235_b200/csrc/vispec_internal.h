@@ -58,6 +58,10 @@ cudaError_t launch_accept_sampled(const int32_t* draft_ids, const int32_t* paren
                                   const float* u_accept, const float* u_bonus, int B, int N, int V, int32_t* path,
                                   int32_t* accept_len, int32_t* bonus, int* status, cudaStream_t st);
 
+cudaError_t launch_tree_rerank(const int32_t* cand_parent, const int32_t* cand_token, const float* cand_score, int B,
+                               int M, int K, int32_t* parents, int32_t* draft_ids, int32_t* selected, int* status,
+                               cudaStream_t st);
+
 struct AttnArgs {
     const void* q; const void* k; const void* v;
     const int32_t* kv_len; const uint64_t* mask;
