@@ -53,6 +53,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context: 0 automatic, 1 partials + merge kernel, 2 clusters")
     ap.add_argument("--no-sampled", action="store_true", help="skip the timing of vispec_accept_sampled")
+    ap.add_argument("--paged", type=int, default=0, help="serve the caches from a block pool of this many slots per block (16/32/64/128)")
     ap.add_argument("--with-rope", action="store_true", help="also run vispec_rope_tree_rows before each layer's attention")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying graphs")
     return ap.parse_args()
@@ -184,6 +185,7 @@ class DeviceWorkload:
         self.scale = 1.0 / math.sqrt(D)
         self.kv_bytes_per_layer = cfg.kv_bytes_per_layer(tree["kv_len"])
         self.with_rope = False
+        self.page_rows = 0
 
     def enable_rope(self, tree, theta):
         """Also rotate the tree rows and write them into the cache before each layer's attention (the step that
@@ -199,6 +201,26 @@ class DeviceWorkload:
         self.theta = theta
         self.with_rope = True
 
+    def enable_paging(self, page_rows):
+        """Re-home every layer's cache in a block pool [num_blocks, Hkv, page_rows, D] with the blocks in a seeded
+        random order (what a serving stack's allocator leaves behind) and serve the step through the *_paged calls."""
+        torch, cfg = self.torch, self.cfg
+        B, Hkv, S_max, D = self.k[0].shape
+        per = S_max // page_rows
+        g = torch.Generator(device="cpu").manual_seed(4321)
+        perm = torch.randperm(B * per, generator=g).to(self.dev)
+        self.block_table = perm.view(B, per).to(torch.int32).contiguous()
+        for l in range(self.L):
+            pools = []
+            for c in (self.k[l], self.v[l]):
+                blocks = c.view(B, Hkv, per, page_rows, D).permute(0, 2, 1, 3, 4).reshape(B * per, Hkv, page_rows, D)
+                pool = torch.empty(blocks.shape, dtype=blocks.dtype, device=blocks.device)
+                pool[perm] = blocks
+                pools.append(pool)
+            self.k[l], self.v[l] = pools
+            self.ctx.cache_register_paged(l, self.k[l], self.v[l])
+        self.page_rows = page_rows
+
     def _pre(self):
         self.ctx.tree_mask_build(self.parents, self.mask, self.depth)
 
@@ -207,7 +229,11 @@ class DeviceWorkload:
             if self.with_rope:
                 self.ctx.rope_tree_rows(l, self.q[l], self.k_new[l], self.v_new[l], self.positions, self.kv_len,
                                         self.theta)
-            self.ctx.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
+            if self.page_rows:
+                self.ctx.tree_verify_attn_paged(l, self.q[l], self.kv_len, self.block_table, self.mask, self.scale,
+                                                self.out[l])
+            else:
+                self.ctx.tree_verify_attn(l, self.q[l], self.kv_len, self.mask, self.scale, self.out[l])
 
     def _probe(self):
         for l in range(self.L):
@@ -215,6 +241,10 @@ class DeviceWorkload:
 
     def _post(self):
         # acceptance and commit in one launch; kv_len itself is left as it was so that every step sees the same workload
+        if self.page_rows:
+            self.ctx.accept(self.draft, self.target, self.parents, self.path, self.alen, self.bonus)
+            self.ctx.kv_compact_paged(0, self.L, self.path, self.alen, self.kv_len, self.block_table, self.new_len)
+            return
         self.ctx.accept_commit(0, self.L, self.draft, self.target, self.parents, self.kv_len, self.path, self.alen,
                                self.bonus, self.new_len)
 
@@ -381,7 +411,9 @@ def main():
         from paper_2509_15235_b200 import binding
         wl.ctx.ctx_set_option(binding.OPT_SPLIT_FORM, args.split_form)
     L = wl.L
-    if args.with_rope:
+    if args.paged:
+        wl.enable_paging(args.paged)
+    if args.with_rope and not args.paged:
         wl.enable_rope(tree, 1e6 if cfg.name.startswith("qwen") else 1e4)
 
     def barrier():
@@ -424,7 +456,7 @@ def main():
 
     # ---- streaming-read probe: the same K/V rows through the same TMA rings, no arithmetic (context for the roofline) ----
     read_probe = None
-    if rank == 0 and cfg.D == 128 and cfg.B <= 32:
+    if rank == 0 and cfg.D == 128 and cfg.B <= 32 and not args.paged:
         torch = wl.torch
         g = torch.cuda.CUDAGraph()
         wl._probe()
@@ -504,7 +536,7 @@ def main():
 
     # ---- end-to-end timing (host buffers in, host results out) ----
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.paged:     # the host-buffer step writes the tree rows into contiguous caches
         hs = HostStep(wl, tree, per_layer)
         for _ in range(3):
             hs.step()
@@ -537,7 +569,7 @@ def main():
                    "kv_bytes_per_layer": wl.kv_bytes_per_layer,
                    "l2": f"inputs larger than L2: {L} layers x {wl.kv_bytes_per_layer / 1e6:.1f} MB rotate, no flush",
                    "launch": "plain C-ABI calls" if args.no_graph else "C-ABI calls captured once, replayed as 3 CUDA graphs per step",
-                   "rope_tree_rows": bool(args.with_rope),
+                   "rope_tree_rows": bool(args.with_rope), "paged_block_rows": args.paged,
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
         "attn_us_per_layer": attn_s * 1e6,

@@ -178,6 +178,37 @@ int vispec_tree_verify_attn_static(const void* q, const void* k_cache, const voi
                                    int Hq, int Hkv, int D, int S_max, float scale, void* out,
                                    float* lse, int* status_word, void* stream);
 
+/* Paged cache (the paper's runtime uses one pre-allocated cache per sequence, App. A; a serving stack shares a
+ * pool of fixed-size blocks between sequences instead - same arithmetic, another layout).
+ *   k_pool, v_pool: bf16 [num_blocks, Hkv, page_rows, D] (device, 128-byte aligned, caller-owned), page_rows in
+ *   {16, 32, 64, 128}, D = 128 only (E_UNSUPPORTED otherwise).  Registering a layer replaces what was registered
+ *   for it before, paged or not.  A paged layer is served by the *_paged calls only (the others answer
+ *   E_UNSUPPORTED for it, and the *_paged calls answer E_UNSUPPORTED for a contiguous layer).
+ * Host errors: E_NULL, E_RANGE (layer), E_ALIGN, E_UNSUPPORTED, E_SHAPE. */
+int vispec_cache_register_paged(vispec_ctx* ctx, int layer, void* k_pool, void* v_pool, int num_blocks, int page_rows);
+
+/* vispec_tree_verify_attn on a paged layer.  block_table [B, table_stride] int32 (device): entry i of row b is
+ * the pool block that holds logical slots [i * page_rows, (i + 1) * page_rows) of sequence b; only the entries of
+ * blocks that start below kv_len[b] + N are read.  Logical slots mean what they mean in the contiguous call
+ * (prefix at [0, kv_len), tree rows at kv_len + i); capacity is table_stride * page_rows slots (a sequence with
+ * kv_len + N beyond it is skipped: zero output, -inf lse, status VISPEC_E_RANGE).  A table entry outside
+ * [0, num_blocks) reads as zeros and sets the status word VISPEC_E_RANGE; nothing faults.  The table, like
+ * kv_len and the committed prefix, must not be written by the kernel that precedes this call on the stream.
+ * Everything else (q, tree_mask, scale, out, lse, workspace, accuracy) as in vispec_tree_verify_attn.
+ * Host errors: E_NULL, E_ALIGN, E_SHAPE, E_RANGE, E_UNREGISTERED, E_UNSUPPORTED (contiguous layer, B > 32,
+ * scale <= 0), E_WORKSPACE. */
+int vispec_tree_verify_attn_paged(vispec_ctx* ctx, int layer, const void* q, const int32_t* kv_len,
+                                  const int32_t* block_table, int table_stride, const uint64_t* tree_mask, int B, int N,
+                                  float scale, void* out, float* lse, void* stream);
+
+/* vispec_kv_compact on paged layers [layer_begin, layer_end): rows move between logical slots kv_len + path[k]
+ * and kv_len + k, each found through block_table (one table serves all layers of the range, which must share
+ * num_blocks and page_rows: E_SHAPE otherwise).  A table entry outside the pool drops that row's move and sets
+ * the status word VISPEC_E_RANGE.  Other arguments and errors as in vispec_kv_compact. */
+int vispec_kv_compact_paged(vispec_ctx* ctx, int layer_begin, int layer_end, const int32_t* path,
+                            const int32_t* accept_len, const int32_t* kv_len, const int32_t* block_table,
+                            int table_stride, int32_t* kv_len_out, int B, int N, void* stream);
+
 /* Rotary position embedding of the tree rows and their placement in the cache: the step just before
  * vispec_tree_verify_attn of the same layer (Sec. 3.2: the target LLM runs unchanged; LLaVA-v1.6 and
  * Qwen2.5-VL rotate q and k by position, pairing element j with element j + D/2).  For node i of sequence b

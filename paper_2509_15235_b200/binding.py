@@ -26,6 +26,7 @@ EXPORTS = [
     "vispec_ctx_set_workspace", "vispec_cache_register", "vispec_tree_mask_build",
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
     "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows", "vispec_accept_sampled", "vispec_tree_rerank",
+    "vispec_cache_register_paged", "vispec_tree_verify_attn_paged", "vispec_kv_compact_paged",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
@@ -71,6 +72,9 @@ def load() -> ctypes.CDLL:
             "vispec_stream_probe": [vp, ci, vp, ci, ci, vp],
             "vispec_accept_sampled": [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp],
             "vispec_tree_rerank": [vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp],
+            "vispec_cache_register_paged": [vp, ci, vp, vp, ci, ci],
+            "vispec_tree_verify_attn_paged": [vp, ci, vp, vp, vp, ci, vp, ci, ci, cf, vp, vp, vp],
+            "vispec_kv_compact_paged": [vp, ci, ci, vp, vp, vp, vp, ci, vp, ci, ci, vp],
             "vispec_rope_tree_rows": [vp, ci, vp, vp, vp, vp, vp, ci, ci, cf, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
@@ -212,6 +216,27 @@ class VerifyContext:
         _check(self.lib.vispec_tree_rerank(self.handle, _ptr(cand_parent), _ptr(cand_token), _ptr(cand_score), B, M, K,
                                            _ptr(parents), _ptr(draft_ids), _ptr(selected), _stream()),
                "vispec_tree_rerank")
+
+    def cache_register_paged(self, layer: int, k_pool: torch.Tensor, v_pool: torch.Tensor) -> None:
+        num_blocks, _, page_rows, _ = k_pool.shape
+        _check(self.lib.vispec_cache_register_paged(self.handle, layer, _ptr(k_pool), _ptr(v_pool), num_blocks, page_rows),
+               "vispec_cache_register_paged")
+        self._caches[layer] = (k_pool, v_pool)   # keep the tensors alive
+
+    def tree_verify_attn_paged(self, layer: int, q: torch.Tensor, kv_len: torch.Tensor, block_table: torch.Tensor,
+                               tree_mask: torch.Tensor, scale: float, out: torch.Tensor,
+                               lse: Optional[torch.Tensor] = None) -> None:
+        B, N = q.shape[0], q.shape[1]
+        _check(self.lib.vispec_tree_verify_attn_paged(self.handle, layer, _ptr(q), _ptr(kv_len), _ptr(block_table),
+                                                      block_table.shape[1], _ptr(tree_mask), B, N, ctypes.c_float(scale),
+                                                      _ptr(out), _ptr(lse), _stream()), "vispec_tree_verify_attn_paged")
+
+    def kv_compact_paged(self, layer_begin: int, layer_end: int, path: torch.Tensor, accept_len: torch.Tensor,
+                         kv_len: torch.Tensor, block_table: torch.Tensor, kv_len_out: Optional[torch.Tensor]) -> None:
+        B, N = path.shape
+        _check(self.lib.vispec_kv_compact_paged(self.handle, layer_begin, layer_end, _ptr(path), _ptr(accept_len),
+                                                _ptr(kv_len), _ptr(block_table), block_table.shape[1], _ptr(kv_len_out),
+                                                B, N, _stream()), "vispec_kv_compact_paged")
 
     def rope_tree_rows(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
                        positions: torch.Tensor, kv_len: torch.Tensor, theta: float) -> None:

@@ -70,7 +70,7 @@ extern "C" int vispec_tree_verify_attn_static(const void* q, const void* k_cache
     if (rc != VISPEC_OK) return rc;
     const DeviceSetup& s = g_setup[dev];
 
-    vispec::AttnArgs a;
+    vispec::AttnArgs a = {};
     a.q = q; a.k = k_cache; a.v = v_cache; a.kv_len = kv_len; a.mask = tree_mask; a.out = out; a.lse = lse;
     a.B = B; a.N = N; a.Hq = Hq; a.Hkv = Hkv; a.D = D; a.S_max = S_max; a.scale = scale;
     a.ws = s.scratch; a.ws_bytes = VISPEC_STATIC_SCRATCH_BYTES;

@@ -95,7 +95,8 @@ struct Sched {
     int len[kMaxB];        // committed length S of sequence b
     int units;             // units with at least one step
 };
-constexpr int SMEM_TOTAL = SMEM_SCHED + (int)sizeof(Sched);
+constexpr int SMEM_TABRING = SMEM_SCHED + ((int)sizeof(Sched) + 15) / 16 * 16;   // 8 steps x 8 block numbers (paged cache)
+constexpr int SMEM_TOTAL = SMEM_TABRING + 256;
 constexpr int SMEM_ALLOC = SMEM_TOTAL;                         // the base must come out 1024-byte aligned (checked)
 static_assert(SMEM_ALLOC <= 232448, "over the 227 KB a CTA may have");
 
@@ -390,9 +391,91 @@ struct SegIter {
     }
 };
 
-template <bool PAIR, bool CL>
+// ---- producer of a paged segment ---------------------------------------------------------------------
+// Paged cache: a step's 128 slots are 128 / page_rows pool blocks, each its own box.  The block numbers travel
+// from the table to a small ring in shared memory by asynchronous 4-byte copies issued six steps ahead of their
+// use: a plain load held in a register that long would share a scoreboard with the waits and copies in between
+// and stall them for its whole latency.  Blocks that start at or past kv_len + N are not fetched: their table
+// entries need not exist, and the rows they would fill are masked like any slot past the end.  Not inlined, so
+// that it stays out of the kernel's register budget, and everything by value, so that the caller's counters stay in
+// registers.  Runs in one thread.  Returns steps issued in full | K-only step << 28 | a wait gave up << 29 |
+// has waited for the preceding kernel << 30.
+constexpr int kTabRing = 8, kTabAhead = 6;     // steps held in the ring / steps a copy is issued ahead
+// pool [num_blocks][Hkv][page_rows][D]; block_table[b][i] = pool block of logical slots [i * page_rows, (i + 1) * page_rows)
+struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N; int* status; };
+__device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensorMap* k_map, const CUtensorMap* v_map,
+                                               int b, int kvh, int st0, int n, int S, uint32_t base, uint32_t bars,
+                                               uint32_t ring, volatile int* abort_flag, uint64_t pol, int it,
+                                               bool waited) {
+    auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+    const int nsub = STEP / p.page_rows;
+    const uint32_t sub_bytes = (uint32_t)p.page_rows * 128u;
+    const int32_t* trow = p.block_table + (size_t)b * p.table_stride;
+    const int total = S + p.N;
+    auto issue = [&](int t) {                  // one group per step, empty past the segment's end
+        if (t < n) {
+            for (int j = 0; j < nsub; ++j) {
+                const int blk = (st0 + t) * nsub + j;
+                if (blk * p.page_rows < total)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(ring + 4u * (uint32_t)((t % kTabRing) * 8 + j)), "l"(trow + blk) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    for (int t = 0; t < kTabAhead; ++t) issue(t);
+    uint32_t fail = 0;
+    int t = 0;
+    for (; t < n; ++t, ++it) {
+        issue(t + kTabAhead);
+        asm volatile("cp.async.wait_group %0;" ::"n"(kTabAhead) : "memory");     // the group of step t has landed
+        const int tok = (st0 + t) * STEP;
+        if (!waited && tok + STEP > S) { pdl_wait(); waited = true; }   // the tree's rows come from the preceding kernel
+        int e[8];
+        int nload = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            e[j] = -1;
+            if (j < nsub && tok + j * p.page_rows < total) {
+                ++nload;
+                asm volatile("ld.shared.s32 %0, [%1];" : "=r"(e[j]) : "r"(ring + 4u * (uint32_t)((t % kTabRing) * 8 + j)) : "memory");
+                if (e[j] < 0 || e[j] >= p.num_blocks) {                  // out of the pool: reported, read as zeros
+                    if (p.status) atomicCAS(p.status, 0, VISPEC_E_RANGE);
+                    e[j] = -1;
+                }
+            }
+        }
+        const int sk = it % NSK, sv = it % NSV;
+        if (!mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag)) { fail = 2u << 28; break; }
+        mbar_expect_tx(bar(B_KFULL + sk), (uint32_t)nload * sub_bytes * 2u);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < nload) {
+                const int z = e[j] >= 0 ? e[j] * p.Hkv + kvh : -1;
+                tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + j * sub_bytes, k_map, bar(B_KFULL + sk), 0, 0, z, pol);
+                tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES + j * sub_bytes, k_map, bar(B_KFULL + sk), 64, 0, z, pol);
+            }
+        }
+        if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { fail = 3u << 28; break; }
+        mbar_expect_tx(bar(B_VFULL + sv), (uint32_t)nload * sub_bytes * 2u);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < nload) {
+                const int z = e[j] >= 0 ? e[j] * p.Hkv + kvh : -1;
+                tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + j * sub_bytes, v_map, bar(B_VFULL + sv), 0, 0, z, pol);
+                tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES + j * sub_bytes, v_map, bar(B_VFULL + sv), 64, 0, z, pol);
+            }
+        }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");                     // nothing of this segment stays in flight
+    return (uint32_t)t | fail | (waited ? 1u << 30 : 0u);
+}
+
+// PAGED instantiations carry the paged producer; the others are compiled without it (its call sites cost the
+// contiguous kernels registers they do not have to spare).
+template <bool PAIR, bool CL, bool PAGED>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const Tc5Params p) {
+attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const Tc5Params p,
+                const PagedArgs pa) {
     constexpr int ROWS = PAIR ? 64 : 128;      // distinct query rows per CTA
     constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
     extern __shared__ __align__(1024) unsigned char sm[];
@@ -476,7 +559,16 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             bool ok = true;
             SegIter si = make_iter();
             Seg sg;
-            while (ok && si.next(sg)) {
+            if constexpr (PAGED) {
+                while (ok && si.next(sg)) {
+                    const uint32_t r = produce_paged(pa, &k_map, &v_map, sg.b, sg.kvh, sg.st0, sg.n, sg.S, base, bars, base + SMEM_TABRING, abort_flag, pol, it, waited);
+                    const int done = (int)(r & 0x0fffffffu);
+                    it += done; nv += done; nk += done + (int)((r >> 28) & 1u);
+                    ok = !((r >> 29) & 1u);
+                    waited = (r >> 30) & 1u;
+                }
+            }
+            while (!PAGED && ok && si.next(sg)) {
                 const int bh = sg.b * p.Hkv + sg.kvh;
                 for (int t = 0; t < sg.n; ++t, ++it) {
                     const int tok = (sg.st0 + t) * STEP;
@@ -1208,8 +1300,8 @@ static int query_max_clusters(bool pair, int k) {
     attr[0].val.clusterDim.x = k; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int n = 0;
-    cudaError_t e = pair ? cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<true, true>, &cfg)
-                         : cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<false, true>, &cfg);
+    cudaError_t e = pair ? cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<true, true, false>, &cfg)
+                         : cudaOccupancyMaxActiveClusters(&n, attn_tc5_kernel<false, true, false>, &cfg);
     if (e != cudaSuccess) { cudaGetLastError(); return 0; }
     return n;
 }
@@ -1243,14 +1335,15 @@ bool attn_tc5_supports(const AttnArgs& a) {
 }
 
 cudaError_t init_attn_tc5() {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc5_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc5_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc5_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    const void* kernels[8] = {(const void*)attn_tc5_kernel<true, false, false>, (const void*)attn_tc5_kernel<false, false, false>,
+                              (const void*)attn_tc5_kernel<true, true, false>, (const void*)attn_tc5_kernel<false, true, false>,
+                              (const void*)attn_tc5_kernel<true, false, true>, (const void*)attn_tc5_kernel<false, false, true>,
+                              (const void*)attn_tc5_kernel<true, true, true>, (const void*)attn_tc5_kernel<false, true, true>};
+    for (const void* k : kernels) {
+        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+    }
     for (int k = 1; k <= 8; ++k) { g_max_clusters[0][k] = query_max_clusters(false, k); g_max_clusters[1][k] = query_max_clusters(true, k); }
     if (getenv("VISPEC_DEBUG")) for (int k = 1; k <= 8; ++k) fprintf(stderr, "vispec: cluster size %d: %d (rows > 64) / %d (rows <= 64) co-resident clusters\n", k, g_max_clusters[0][k], g_max_clusters[1][k]);
     // The merge blocks must be able to join an SM that an attention CTA has configured for maximum shared memory.
@@ -1270,7 +1363,7 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     const int ck = tc5_cluster_size(a, units);
     const int grid = ck > 0 ? units * ck : (int)(t_max < a.sm_count ? t_max : a.sm_count);
 
-    Tc5Params p;
+    Tc5Params p = {};
     p.q = (const __nv_bfloat16*)a.q; p.kv_len = a.kv_len; p.mask = a.mask;
     p.out = (__nv_bfloat16*)a.out; p.lse = a.lse;
     unsigned char* ws = (unsigned char*)a.ws + kCounterBytes;
@@ -1286,16 +1379,21 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     p.trace_idx = 0;
 #endif
     cudaError_t err;
+    const bool paged = a.page_rows != 0;
+    const PagedArgs pa = {a.block_table, a.table_stride, a.page_rows, a.num_blocks, a.Hkv, a.N, a.status};
+    auto launch_attn = [&](auto kernel, int cluster) {
+        return launch_pdl(kernel, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, cluster, *a.k_map, *a.v_map, p, pa);
+    };
     if (ck > 0) {
         // cluster form: the CTAs of a unit merge their partials through distributed shared memory; one launch
-        err = pair ? launch_pdl(attn_tc5_kernel<true, true>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, ck, *a.k_map, *a.v_map, p)
-                   : launch_pdl(attn_tc5_kernel<false, true>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, ck, *a.k_map, *a.v_map, p);
+        err = paged ? (pair ? launch_attn(attn_tc5_kernel<true, true, true>, ck) : launch_attn(attn_tc5_kernel<false, true, true>, ck))
+                    : (pair ? launch_attn(attn_tc5_kernel<true, true, false>, ck) : launch_attn(attn_tc5_kernel<false, true, false>, ck));
         if (err != cudaSuccess) return err;
         ++*n_launches;
         return cudaSuccess;
     }
-    err = pair ? launch_pdl(attn_tc5_kernel<true, false>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, 0, *a.k_map, *a.v_map, p)
-               : launch_pdl(attn_tc5_kernel<false, false>, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, 0, *a.k_map, *a.v_map, p);
+    err = paged ? (pair ? launch_attn(attn_tc5_kernel<true, false, true>, 0) : launch_attn(attn_tc5_kernel<false, false, true>, 0))
+                : (pair ? launch_attn(attn_tc5_kernel<true, false, false>, 0) : launch_attn(attn_tc5_kernel<false, false, false>, 0));
     if (err != cudaSuccess) return err;
     ++*n_launches;
     err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p)

@@ -145,7 +145,8 @@ constexpr int kCompactRows = 16;
 __global__ void __launch_bounds__(256)
 kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const int32_t* __restrict__ path,
                   const int32_t* __restrict__ accept_len, const int32_t* __restrict__ kv_len,
-                  int32_t* __restrict__ kv_len_out, int N, int Hkv, int D, int S_max, int* status) {
+                  int32_t* __restrict__ kv_len_out, int N, int Hkv, int D, int S_max, int* status,
+                  const int32_t* __restrict__ block_table, int table_stride, int page_rows, int num_blocks) {
     __shared__ uint4 stage[2][kCompactRows][16];   // up to 256 B per row (D = 128)
     __shared__ int32_t src_row[kCompactRows];
     const int layer = layer_begin + blockIdx.z, b = blockIdx.y, h = blockIdx.x;
@@ -159,9 +160,17 @@ kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const i
     const int tensor = threadIdx.x >> 7;             // 0: K, 1: V
     const int r = (threadIdx.x & 127) >> 3;          // row of the pass, 0..15
     const int c0 = threadIdx.x & 7;                  // this thread moves chunks c0 and c0 + 8
-    uint4* base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]) +
-                  ((size_t)b * Hkv + h) * (size_t)S_max * chunks;
+    uint4* const tensor_base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]);
+    uint4* base = tensor_base + ((size_t)b * Hkv + h) * (size_t)S_max * chunks;
     bool bad = false;
+    // Paged cache (pool [num_blocks][Hkv][page_rows][D]): a logical slot's row is found through the block table; a
+    // table entry outside the pool drops the move and is reported.
+    auto row_of = [&](int slot) -> uint4* {
+        if (!block_table) return base + (size_t)slot * chunks;
+        const int blk = block_table[(size_t)b * table_stride + slot / page_rows];
+        if (blk < 0 || blk >= num_blocks) { bad = true; return nullptr; }
+        return tensor_base + (((size_t)blk * Hkv + h) * page_rows + slot % page_rows) * (size_t)chunks;
+    };
     for (int k0 = 0; k0 < L; k0 += kCompactRows) {
         if (threadIdx.x < kCompactRows) {
             const int k = k0 + threadIdx.x;
@@ -171,14 +180,15 @@ kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const i
         }
         __syncthreads();
         const int s = src_row[r];
-        if (s >= 0) {
-            const uint4* src = base + (size_t)(S + s) * chunks;
+        const uint4* src = s >= 0 ? row_of(S + s) : nullptr;
+        uint4* dst = s >= 0 ? row_of(S + k0 + r) : nullptr;
+        const bool move = src && dst;
+        if (move) {
             if (c0 < chunks) stage[tensor][r][c0] = src[c0];
             if (c0 + 8 < chunks) stage[tensor][r][c0 + 8] = src[c0 + 8];
         }
         __syncthreads();
-        if (s >= 0) {
-            uint4* dst = base + (size_t)(S + k0 + r) * chunks;
+        if (move) {
             if (c0 < chunks) dst[c0] = stage[tensor][r][c0];
             if (c0 + 8 < chunks) dst[c0 + 8] = stage[tensor][r][c0 + 8];
         }
@@ -191,11 +201,12 @@ kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const i
 cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int layer_end,
                               const int32_t* path, const int32_t* accept_len, const int32_t* kv_len,
                               int32_t* kv_len_out, int B, int N, int Hkv, int D, int S_max, int* status,
-                              cudaStream_t st) {
+                              cudaStream_t st, const int32_t* block_table, int table_stride, int page_rows,
+                              int num_blocks) {
     if (B == 0 || layer_end <= layer_begin) return cudaSuccess;
     dim3 grid(Hkv, B, layer_end - layer_begin);
     kv_compact_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, path, accept_len, kv_len, kv_len_out,
-                                            N, Hkv, D, S_max, status);
+                                            N, Hkv, D, S_max, status, block_table, table_stride, page_rows, num_blocks);
     return cudaGetLastError();
 }
 

@@ -91,6 +91,8 @@ int vispec_ctx_create(vispec_ctx** out, const vispec_shape* s, int device) {
     const char* fg = std::getenv("VISPEC_FORCE_GENERIC");
     c->force_generic = fg && fg[0] == '1';
     c->k_map.resize(s->layers);
+    c->page_rows.assign(s->layers, 0);
+    c->num_blocks.assign(s->layers, 0);
     c->v_map.resize(s->layers);
     *out = c;
     return VISPEC_OK;
@@ -161,6 +163,42 @@ int vispec_cache_register(vispec_ctx* c, int layer, void* k_cache, void* v_cache
         return VISPEC_E_CUDA;
     c->h_k[layer] = k_cache;
     c->h_v[layer] = v_cache;
+    c->page_rows[layer] = 0;
+    c->num_blocks[layer] = 0;
+    return VISPEC_OK;
+}
+
+int vispec_cache_register_paged(vispec_ctx* c, int layer, void* k_pool, void* v_pool, int num_blocks, int page_rows) {
+    if (!c || !k_pool || !v_pool) return VISPEC_E_NULL;
+    if (layer < 0 || layer >= c->shape.layers) return VISPEC_E_RANGE;
+    if (!aligned(k_pool, 128) || !aligned(v_pool, 128)) return VISPEC_E_ALIGN;
+    const vispec_shape& s = c->shape;
+    if (s.D != 128) return VISPEC_E_UNSUPPORTED;
+    if (num_blocks < 1 || (page_rows != 16 && page_rows != 32 && page_rows != 64 && page_rows != 128)) return VISPEC_E_SHAPE;
+    if ((long long)num_blocks * s.Hkv >= (1ll << 31)) return VISPEC_E_SHAPE;
+    // 3-D view (d, slot in block, block*head) of a [num_blocks,Hkv,page_rows,D] bf16 pool; one box = 64 d-columns x one
+    // block's slots of one head.  A block number outside the pool reads as zero.
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return VISPEC_E_CUDA;
+    const cuuint64_t dims[3] = {(cuuint64_t)s.D, (cuuint64_t)page_rows, (cuuint64_t)num_blocks * s.Hkv};
+    const cuuint64_t strides[2] = {(cuuint64_t)s.D * 2, (cuuint64_t)page_rows * s.D * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)page_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    void* ptrs[2] = {k_pool, v_pool};
+    CUtensorMap* maps[2] = {&c->k_map[layer], &c->v_map[layer]};
+    for (int t = 0; t < 2; ++t) {
+        CUresult r = enc(maps[t], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ptrs[t], dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return VISPEC_E_CUDA;
+    }
+    void* pair[2] = {k_pool, v_pool};
+    if (cudaMemcpy(c->d_cache_ptrs + 2 * layer, pair, sizeof(pair), cudaMemcpyHostToDevice) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    c->h_k[layer] = k_pool;
+    c->h_v[layer] = v_pool;
+    c->page_rows[layer] = page_rows;
+    c->num_blocks[layer] = num_blocks;
     return VISPEC_OK;
 }
 
@@ -185,8 +223,9 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
     if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
     if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
     if ((k_cache && k_cache != c->h_k[layer]) || (v_cache && v_cache != c->h_v[layer])) return VISPEC_E_UNREGISTERED;
+    if (c->page_rows[layer]) return VISPEC_E_UNSUPPORTED;     // a paged layer goes through vispec_tree_verify_attn_paged
     if (!c->ws) return VISPEC_E_WORKSPACE;
-    AttnArgs a;
+    AttnArgs a = {};
     a.q = q; a.k = c->h_k[layer]; a.v = c->h_v[layer];
     a.kv_len = kv_len; a.mask = tree_mask; a.out = out; a.lse = lse;
     a.B = B; a.N = N; a.Hq = s.Hq; a.Hkv = s.Hkv; a.D = s.D; a.S_max = s.S_max;
@@ -202,6 +241,62 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
     return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
 }
 
+int vispec_tree_verify_attn_paged(vispec_ctx* c, int layer, const void* q, const int32_t* kv_len,
+                                  const int32_t* block_table, int table_stride, const uint64_t* tree_mask, int B, int N,
+                                  float scale, void* out, float* lse, void* stream) {
+    if (!c || !q || !kv_len || !block_table || !tree_mask || !out) return VISPEC_E_NULL;
+    if (!aligned(q, 16) || !aligned(out, 16)) return VISPEC_E_ALIGN;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max || table_stride < 1) return VISPEC_E_SHAPE;
+    if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
+    if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
+    if (!c->page_rows[layer]) return VISPEC_E_UNSUPPORTED;
+    if ((long long)table_stride * c->page_rows[layer] > (1ll << 30)) return VISPEC_E_SHAPE;
+    if (!c->ws) return VISPEC_E_WORKSPACE;
+    if (B == 0) return VISPEC_OK;
+    AttnArgs a = {};
+    a.q = q; a.k = c->h_k[layer]; a.v = c->h_v[layer];
+    a.kv_len = kv_len; a.mask = tree_mask; a.out = out; a.lse = lse;
+    a.B = B; a.N = N; a.Hq = s.Hq; a.Hkv = s.Hkv; a.D = s.D;
+    a.S_max = table_stride * c->page_rows[layer];
+    a.scale = scale; a.ws = c->ws; a.ws_bytes = c->ws_bytes; a.status = c->d_status;
+    a.sm_count = c->sm_count;
+    a.early_prefetch = c->early_prefetch;
+    a.tc5_path = c->tc5_path;
+    a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
+    a.block_table = block_table; a.table_stride = table_stride;
+    a.page_rows = c->page_rows[layer]; a.num_blocks = c->num_blocks[layer];
+    if (!attn_tc5_supports(a)) return VISPEC_E_UNSUPPORTED;   // B <= 32, scale > 0, workspace large enough for the table's capacity
+    int n = 0;
+    cudaError_t err = launch_attn_tc5(a, (cudaStream_t)stream, &n);
+    c->launches += n;
+    return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
+}
+
+int vispec_kv_compact_paged(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* path,
+                            const int32_t* accept_len, const int32_t* kv_len, const int32_t* block_table,
+                            int table_stride, int32_t* kv_len_out, int B, int N, void* stream) {
+    if (!c || !path || !accept_len || !kv_len || !block_table) return VISPEC_E_NULL;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max || table_stride < 1) return VISPEC_E_SHAPE;
+    if (layer_begin < 0 || layer_end > s.layers || layer_begin > layer_end) return VISPEC_E_RANGE;
+    if (kv_len_out == kv_len) return VISPEC_E_SHAPE;
+    if (layer_begin == layer_end) return VISPEC_OK;
+    const int pr = c->page_rows[layer_begin], nb = c->num_blocks[layer_begin];
+    for (int l = layer_begin; l < layer_end; ++l) {
+        if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
+        if (!c->page_rows[l]) return VISPEC_E_UNSUPPORTED;
+        if (c->page_rows[l] != pr || c->num_blocks[l] != nb) return VISPEC_E_SHAPE;   // one table serves every layer
+    }
+    if ((long long)table_stride * pr > (1ll << 30)) return VISPEC_E_SHAPE;
+    if (launch_kv_compact(c->d_cache_ptrs, layer_begin, layer_end, path, accept_len, kv_len, kv_len_out, B, N, s.Hkv,
+                          s.D, table_stride * pr, c->d_status, (cudaStream_t)stream, block_table, table_stride, pr,
+                          nb) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
 int vispec_rope_tree_rows(vispec_ctx* c, int layer, void* q, const void* k_new, const void* v_new,
                           const int32_t* positions, const int32_t* kv_len, int B, int N, float theta, void* stream) {
     if (!c || !q || !k_new || !v_new || !positions || !kv_len) return VISPEC_E_NULL;
@@ -210,6 +305,7 @@ int vispec_rope_tree_rows(vispec_ctx* c, int layer, void* q, const void* k_new, 
     if (B < 0 || B > s.B_max || N < 1 || N > s.N_max || !(theta > 1.f)) return VISPEC_E_SHAPE;
     if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
     if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
+    if (c->page_rows[layer]) return VISPEC_E_UNSUPPORTED;
     if (launch_rope_rows(q, k_new, v_new, positions, kv_len, c->h_k[layer], c->h_v[layer], theta, B, N, s.Hq, s.Hkv,
                          s.D, s.S_max, c->d_status, (cudaStream_t)stream) != cudaSuccess)
         return VISPEC_E_CUDA;
@@ -224,6 +320,7 @@ int vispec_stream_probe(vispec_ctx* c, int layer, const int32_t* kv_len, int B, 
     if (s.D != 128) return VISPEC_E_UNSUPPORTED;
     if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
     if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
+    if (c->page_rows[layer]) return VISPEC_E_UNSUPPORTED;
     AttnArgs a = {};
     a.k = c->h_k[layer]; a.v = c->h_v[layer]; a.kv_len = kv_len;
     a.B = B; a.N = N; a.Hq = s.Hq; a.Hkv = s.Hkv; a.D = s.D; a.S_max = s.S_max;
@@ -280,8 +377,10 @@ int vispec_kv_compact(vispec_ctx* c, int layer_begin, int layer_end, const int32
     if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
     if (layer_begin < 0 || layer_end > s.layers || layer_begin > layer_end) return VISPEC_E_RANGE;
     if (kv_len_out == kv_len) return VISPEC_E_SHAPE;
-    for (int l = layer_begin; l < layer_end; ++l)
+    for (int l = layer_begin; l < layer_end; ++l) {
         if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
+        if (c->page_rows[l]) return VISPEC_E_UNSUPPORTED;
+    }
     if (launch_kv_compact(c->d_cache_ptrs, layer_begin, layer_end, path, accept_len, kv_len, kv_len_out, B, N,
                           s.Hkv, s.D, s.S_max, c->d_status, (cudaStream_t)stream) != cudaSuccess)
         return VISPEC_E_CUDA;
@@ -297,8 +396,10 @@ int vispec_accept_commit(vispec_ctx* c, int layer_begin, int layer_end, const in
     if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
     if (layer_begin < 0 || layer_end > s.layers || layer_begin > layer_end) return VISPEC_E_RANGE;
     if (kv_len_out == kv_len) return VISPEC_E_SHAPE;
-    for (int l = layer_begin; l < layer_end; ++l)
+    for (int l = layer_begin; l < layer_end; ++l) {
         if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
+        if (c->page_rows[l]) return VISPEC_E_UNSUPPORTED;
+    }
     if (layer_end == layer_begin) {
         // nothing to commit: plain acceptance
         if (launch_accept(draft_ids, target_ids, parents, B, N, path, accept_len, bonus, c->d_status,

@@ -16,6 +16,7 @@ struct vispec_ctx {
     void** d_cache_ptrs = nullptr;  // device table [layers][2]: k_cache, v_cache
     std::vector<void*> h_k, h_v;    // host copy of the registered pointers
     std::vector<CUtensorMap> k_map, v_map;  // TMA descriptors per layer (D == 128 only)
+    std::vector<int> page_rows, num_blocks; // per layer: slots per pool block (0 = contiguous cache), pool blocks
     void* ws = nullptr;             // caller-owned workspace
     size_t ws_bytes = 0;
     uint64_t launches = 0;
@@ -43,7 +44,8 @@ cudaError_t launch_accept(const int32_t* draft, const int32_t* target, const int
 cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int layer_end,
                               const int32_t* path, const int32_t* accept_len, const int32_t* kv_len,
                               int32_t* kv_len_out, int B, int N, int Hkv, int D, int S_max, int* status,
-                              cudaStream_t st);
+                              cudaStream_t st, const int32_t* block_table = nullptr, int table_stride = 0,
+                              int page_rows = 0, int num_blocks = 0);
 
 cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int layer_end, const int32_t* draft,
                                  const int32_t* target, const int32_t* parents, const int32_t* kv_len,
@@ -74,6 +76,9 @@ struct AttnArgs {
     bool early_prefetch;   // committed-prefix tiles may be read before the preceding kernel has completed
     int tc5_path;          // 0 automatic, 1 partials in global memory + merge kernel, 2 clusters where possible
     const CUtensorMap* k_map; const CUtensorMap* v_map;
+    // paged cache (page_rows != 0): pool blocks of page_rows slots, block_table [B][table_stride]; S_max is then
+    // table_stride * page_rows
+    const int32_t* block_table; int table_stride, page_rows, num_blocks;
 };
 // Generic split-KV kernel on warp-level tensor-core instructions (any supported shape).
 cudaError_t init_attn_generic();   // once per device, with that device current
