@@ -392,34 +392,33 @@ struct SegIter {
 };
 
 // ---- producer of a paged segment ---------------------------------------------------------------------
-// Paged cache: a step's 128 slots are 128 / page_rows pool blocks, each its own box.  The block numbers travel
-// from the table to a small ring in shared memory by asynchronous 4-byte copies issued six steps ahead of their
-// use: a plain load held in a register that long would share a scoreboard with the waits and copies in between
-// and stall them for its whole latency.  Blocks that start at or past kv_len + N are not fetched: their table
-// entries need not exist, and the rows they would fill are masked like any slot past the end.  Not inlined, so
-// that it stays out of the kernel's register budget, and everything by value, so that the caller's counters stay in
-// registers.  Runs in one thread.  Returns steps issued in full | K-only step << 28 | a wait gave up << 29 |
-// has waited for the preceding kernel << 30.
+// Paged cache: a step's 128 slots are 128 / page_rows pool blocks, each its own box.  Run by the whole producer
+// warp: lane j owns block j of every step - its table entry and its four copies (two d-halves of K and of V) -
+// so that one instruction issues the copies of all the step's blocks; lane 0 alone waits for the free stage and
+// posts the expected byte count.  The block numbers travel from the table to a small ring in shared memory by
+// asynchronous 4-byte copies issued six steps ahead of their use: a plain load held in a register that long would
+// share a scoreboard with the waits and copies in between and stall them for its whole latency.  Blocks that start
+// at or past kv_len + N are not fetched: their table entries need not exist, and the rows they would fill are
+// masked like any slot past the end.  Not inlined, so that it stays out of the kernel's register budget, and
+// everything by value, so that the caller's counters stay in registers.  Returns steps issued in full | K-only
+// step << 28 | a wait gave up << 29 | has waited for the preceding kernel << 30 (the same in every lane).
 constexpr int kTabRing = 8, kTabAhead = 6;     // steps held in the ring / steps a copy is issued ahead
 // pool [num_blocks][Hkv][page_rows][D]; block_table[b][i] = pool block of logical slots [i * page_rows, (i + 1) * page_rows)
 struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N; int* status; };
 __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensorMap* k_map, const CUtensorMap* v_map,
                                                int b, int kvh, int st0, int n, int S, uint32_t base, uint32_t bars,
                                                uint32_t ring, volatile int* abort_flag, uint64_t pol, int it,
-                                               bool waited) {
+                                               bool waited, int lane) {
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     const int nsub = STEP / p.page_rows;
     const uint32_t sub_bytes = (uint32_t)p.page_rows * 128u;
     const int32_t* trow = p.block_table + (size_t)b * p.table_stride;
     const int total = S + p.N;
-    auto issue = [&](int t) {                  // one group per step, empty past the segment's end
-        if (t < n) {
-            for (int j = 0; j < nsub; ++j) {
-                const int blk = (st0 + t) * nsub + j;
-                if (blk * p.page_rows < total)
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(ring + 4u * (uint32_t)((t % kTabRing) * 8 + j)), "l"(trow + blk) : "memory");
-            }
-        }
+    const bool mine = lane < nsub;
+    auto issue = [&](int t) {                  // one group per step and lane, empty where there is nothing to fetch
+        const int blk = (st0 + t) * nsub + lane;
+        if (mine && t < n && blk * p.page_rows < total)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(ring + 4u * (uint32_t)((t % kTabRing) * 8 + lane)), "l"(trow + blk) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
     for (int t = 0; t < kTabAhead; ++t) issue(t);
@@ -427,43 +426,39 @@ __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensor
     int t = 0;
     for (; t < n; ++t, ++it) {
         issue(t + kTabAhead);
-        asm volatile("cp.async.wait_group %0;" ::"n"(kTabAhead) : "memory");     // the group of step t has landed
+        asm volatile("cp.async.wait_group %0;" ::"n"(kTabAhead) : "memory");     // this lane's entry of step t has landed
         const int tok = (st0 + t) * STEP;
         if (!waited && tok + STEP > S) { pdl_wait(); waited = true; }   // the tree's rows come from the preceding kernel
-        int e[8];
-        int nload = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            e[j] = -1;
-            if (j < nsub && tok + j * p.page_rows < total) {
-                ++nload;
-                asm volatile("ld.shared.s32 %0, [%1];" : "=r"(e[j]) : "r"(ring + 4u * (uint32_t)((t % kTabRing) * 8 + j)) : "memory");
-                if (e[j] < 0 || e[j] >= p.num_blocks) {                  // out of the pool: reported, read as zeros
-                    if (p.status) atomicCAS(p.status, 0, VISPEC_E_RANGE);
-                    e[j] = -1;
-                }
-            }
+        const bool load = mine && tok + lane * p.page_rows < total;
+        int z = -1;                                                      // -1: out of the pool, reads as zeros
+        if (load) {
+            int e;
+            asm volatile("ld.shared.s32 %0, [%1];" : "=r"(e) : "r"(ring + 4u * (uint32_t)((t % kTabRing) * 8 + lane)) : "memory");
+            if (e >= 0 && e < p.num_blocks) z = e * p.Hkv + kvh;
+            else if (p.status) atomicCAS(p.status, 0, VISPEC_E_RANGE);
         }
+        const uint32_t tx = (uint32_t)__popc(__ballot_sync(0xffffffffu, load)) * sub_bytes * 2u;
         const int sk = it % NSK, sv = it % NSV;
-        if (!mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag)) { fail = 2u << 28; break; }
-        mbar_expect_tx(bar(B_KFULL + sk), (uint32_t)nload * sub_bytes * 2u);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (j < nload) {
-                const int z = e[j] >= 0 ? e[j] * p.Hkv + kvh : -1;
-                tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + j * sub_bytes, k_map, bar(B_KFULL + sk), 0, 0, z, pol);
-                tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES + j * sub_bytes, k_map, bar(B_KFULL + sk), 64, 0, z, pol);
-            }
+        bool w = true;
+        if (lane == 0) {
+            w = mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag);
+            if (w) mbar_expect_tx(bar(B_KFULL + sk), tx);
         }
-        if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { fail = 3u << 28; break; }
-        mbar_expect_tx(bar(B_VFULL + sv), (uint32_t)nload * sub_bytes * 2u);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (j < nload) {
-                const int z = e[j] >= 0 ? e[j] * p.Hkv + kvh : -1;
-                tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + j * sub_bytes, v_map, bar(B_VFULL + sv), 0, 0, z, pol);
-                tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES + j * sub_bytes, v_map, bar(B_VFULL + sv), 64, 0, z, pol);
-            }
+        w = __shfl_sync(0xffffffffu, w, 0);                              // the byte count is posted before any lane copies
+        if (!w) { fail = 2u << 28; break; }
+        if (load) {
+            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 0, 0, z, pol);
+            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 64, 0, z, pol);
+        }
+        if (lane == 0) {
+            w = mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag);
+            if (w) mbar_expect_tx(bar(B_VFULL + sv), tx);
+        }
+        w = __shfl_sync(0xffffffffu, w, 0);
+        if (!w) { fail = 3u << 28; break; }
+        if (load) {
+            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 0, 0, z, pol);
+            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 64, 0, z, pol);
         }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");                     // nothing of this segment stays in flight
@@ -552,7 +547,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
 
     if (warp == 0) {
         // ================= TMA producer =================
-        if (lane == 0 && active) {
+        if ((PAGED || lane == 0) && active) {        // paged: the whole warp, each lane one block of a step
             const uint64_t pol = l2_evict_first_policy();
             bool waited = !p.early;
             int it = 0, nk = 0, nv = 0;          // steps started; K / V stages issued
@@ -561,7 +556,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             Seg sg;
             if constexpr (PAGED) {
                 while (ok && si.next(sg)) {
-                    const uint32_t r = produce_paged(pa, &k_map, &v_map, sg.b, sg.kvh, sg.st0, sg.n, sg.S, base, bars, base + SMEM_TABRING, abort_flag, pol, it, waited);
+                    const uint32_t r = produce_paged(pa, &k_map, &v_map, sg.b, sg.kvh, sg.st0, sg.n, sg.S, base, bars, base + SMEM_TABRING, abort_flag, pol, it, waited, lane);
                     const int done = (int)(r & 0x0fffffffu);
                     it += done; nv += done; nk += done + (int)((r >> 28) & 1u);
                     ok = !((r >> 29) & 1u);
@@ -589,8 +584,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     ++nv;
                 }
             }
-            if (*abort_flag) {
-                // drain: wait (bounded, fresh timer) until every copy this thread issued has landed
+            if (*abort_flag && lane == 0) {
+                // drain: wait (bounded, fresh timer) until every copy this warp issued has landed
                 volatile int never = 0;
                 for (int u = max(0, nk - NSK); u < nk; ++u) mbar_wait(bar(B_KFULL + u % NSK), (u / NSK) & 1, &never);
                 for (int u = max(0, nv - NSV); u < nv; ++u) mbar_wait(bar(B_VFULL + u % NSV), (u / NSV) & 1, &never);
