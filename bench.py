@@ -226,7 +226,10 @@ class DeviceWorkload:
 
     def _attn(self):
         for l in range(self.L):
-            if self.with_rope:
+            if self.with_rope and self.page_rows:
+                self.ctx.rope_tree_rows_paged(l, self.q[l], self.k_new[l], self.v_new[l], self.positions, self.kv_len,
+                                              self.block_table, self.theta)
+            elif self.with_rope:
                 self.ctx.rope_tree_rows(l, self.q[l], self.k_new[l], self.v_new[l], self.positions, self.kv_len,
                                         self.theta)
             if self.page_rows:
@@ -242,8 +245,8 @@ class DeviceWorkload:
     def _post(self):
         # acceptance and commit in one launch; kv_len itself is left as it was so that every step sees the same workload
         if self.page_rows:
-            self.ctx.accept(self.draft, self.target, self.parents, self.path, self.alen, self.bonus)
-            self.ctx.kv_compact_paged(0, self.L, self.path, self.alen, self.kv_len, self.block_table, self.new_len)
+            self.ctx.accept_commit_paged(0, self.L, self.draft, self.target, self.parents, self.kv_len, self.block_table,
+                                         self.path, self.alen, self.bonus, self.new_len)
             return
         self.ctx.accept_commit(0, self.L, self.draft, self.target, self.parents, self.kv_len, self.path, self.alen,
                                self.bonus, self.new_len)
@@ -413,7 +416,7 @@ def main():
     L = wl.L
     if args.paged:
         wl.enable_paging(args.paged)
-    if args.with_rope and not args.paged:
+    if args.with_rope:
         wl.enable_rope(tree, 1e6 if cfg.name.startswith("qwen") else 1e4)
 
     def barrier():

@@ -209,6 +209,18 @@ int vispec_kv_compact_paged(vispec_ctx* ctx, int layer_begin, int layer_end, con
                             const int32_t* accept_len, const int32_t* kv_len, const int32_t* block_table,
                             int table_stride, int32_t* kv_len_out, int B, int N, void* stream);
 
+/* vispec_accept_commit and vispec_rope_tree_rows on paged layers: the same work, with every logical slot found
+ * through block_table (arguments as in vispec_kv_compact_paged / vispec_tree_verify_attn_paged).  A table entry
+ * outside the pool drops that row's move or placement and sets the status word VISPEC_E_RANGE.  The accepted
+ * range [layer_begin, layer_end) must not be empty here (E_RANGE). */
+int vispec_accept_commit_paged(vispec_ctx* ctx, int layer_begin, int layer_end, const int32_t* draft_ids,
+                               const int32_t* target_ids, const int32_t* parents, const int32_t* kv_len,
+                               const int32_t* block_table, int table_stride, int B, int N, int32_t* path,
+                               int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, void* stream);
+int vispec_rope_tree_rows_paged(vispec_ctx* ctx, int layer, void* q, const void* k_new, const void* v_new,
+                                const int32_t* positions, const int32_t* kv_len, const int32_t* block_table,
+                                int table_stride, int B, int N, float theta, void* stream);
+
 /* Rotary position embedding of the tree rows and their placement in the cache: the step just before
  * vispec_tree_verify_attn of the same layer (Sec. 3.2: the target LLM runs unchanged; LLaVA-v1.6 and
  * Qwen2.5-VL rotate q and k by position, pairing element j with element j + D/2).  For node i of sequence b

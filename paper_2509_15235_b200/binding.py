@@ -27,6 +27,7 @@ EXPORTS = [
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
     "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows", "vispec_accept_sampled", "vispec_tree_rerank",
     "vispec_cache_register_paged", "vispec_tree_verify_attn_paged", "vispec_kv_compact_paged",
+    "vispec_accept_commit_paged", "vispec_rope_tree_rows_paged",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
@@ -75,6 +76,8 @@ def load() -> ctypes.CDLL:
             "vispec_cache_register_paged": [vp, ci, vp, vp, ci, ci],
             "vispec_tree_verify_attn_paged": [vp, ci, vp, vp, vp, ci, vp, ci, ci, cf, vp, vp, vp],
             "vispec_kv_compact_paged": [vp, ci, ci, vp, vp, vp, vp, ci, vp, ci, ci, vp],
+            "vispec_accept_commit_paged": [vp, ci, ci, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp, vp],
+            "vispec_rope_tree_rows_paged": [vp, ci, vp, vp, vp, vp, vp, vp, ci, ci, ci, cf, vp],
             "vispec_rope_tree_rows": [vp, ci, vp, vp, vp, vp, vp, ci, ci, cf, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
@@ -237,6 +240,23 @@ class VerifyContext:
         _check(self.lib.vispec_kv_compact_paged(self.handle, layer_begin, layer_end, _ptr(path), _ptr(accept_len),
                                                 _ptr(kv_len), _ptr(block_table), block_table.shape[1], _ptr(kv_len_out),
                                                 B, N, _stream()), "vispec_kv_compact_paged")
+
+    def accept_commit_paged(self, layer_begin: int, layer_end: int, draft_ids: torch.Tensor, target_ids: torch.Tensor,
+                            parents: torch.Tensor, kv_len: torch.Tensor, block_table: torch.Tensor, path: torch.Tensor,
+                            accept_len: torch.Tensor, bonus: torch.Tensor, kv_len_out: Optional[torch.Tensor]) -> None:
+        B, N = parents.shape
+        _check(self.lib.vispec_accept_commit_paged(self.handle, layer_begin, layer_end, _ptr(draft_ids), _ptr(target_ids),
+                                                   _ptr(parents), _ptr(kv_len), _ptr(block_table), block_table.shape[1],
+                                                   B, N, _ptr(path), _ptr(accept_len), _ptr(bonus), _ptr(kv_len_out),
+                                                   _stream()), "vispec_accept_commit_paged")
+
+    def rope_tree_rows_paged(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                             positions: torch.Tensor, kv_len: torch.Tensor, block_table: torch.Tensor,
+                             theta: float) -> None:
+        B, N = positions.shape
+        _check(self.lib.vispec_rope_tree_rows_paged(self.handle, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(positions),
+                                                    _ptr(kv_len), _ptr(block_table), block_table.shape[1], B, N,
+                                                    ctypes.c_float(theta), _stream()), "vispec_rope_tree_rows_paged")
 
     def rope_tree_rows(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
                        positions: torch.Tensor, kv_len: torch.Tensor, theta: float) -> None:

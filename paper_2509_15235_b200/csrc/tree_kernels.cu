@@ -142,6 +142,19 @@ cudaError_t launch_accept(const int32_t* draft, const int32_t* target, const int
 // ------------------------------------------------------------------------------------------------
 constexpr int kCompactRows = 16;
 
+// Where logical slot `slot` of (sequence b, kv head h) lives, in 16-byte vectors from the tensor's base.
+// Contiguous cache [B,Hkv,S_max,D]: table == nullptr.  Paged pool [num_blocks,Hkv,page_rows,D]: through the block
+// table; -1 if the table entry is outside the pool.
+struct RowMap {
+    const int32_t* table; int table_stride, page_rows, num_blocks;
+    __device__ __forceinline__ long long at(int b, int h, int slot, int Hkv, int S_max, int chunks) const {
+        if (!table) return (((long long)b * Hkv + h) * S_max + slot) * chunks;
+        const int blk = table[(size_t)b * table_stride + slot / page_rows];
+        if (blk < 0 || blk >= num_blocks) return -1;
+        return (((long long)blk * Hkv + h) * page_rows + slot % page_rows) * chunks;
+    }
+};
+
 __global__ void __launch_bounds__(256)
 kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const int32_t* __restrict__ path,
                   const int32_t* __restrict__ accept_len, const int32_t* __restrict__ kv_len,
@@ -161,15 +174,13 @@ kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const i
     const int r = (threadIdx.x & 127) >> 3;          // row of the pass, 0..15
     const int c0 = threadIdx.x & 7;                  // this thread moves chunks c0 and c0 + 8
     uint4* const tensor_base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]);
-    uint4* base = tensor_base + ((size_t)b * Hkv + h) * (size_t)S_max * chunks;
     bool bad = false;
-    // Paged cache (pool [num_blocks][Hkv][page_rows][D]): a logical slot's row is found through the block table; a
-    // table entry outside the pool drops the move and is reported.
+    const RowMap rows = {block_table, table_stride, page_rows, num_blocks};
+    // a table entry outside the pool drops the move and is reported
     auto row_of = [&](int slot) -> uint4* {
-        if (!block_table) return base + (size_t)slot * chunks;
-        const int blk = block_table[(size_t)b * table_stride + slot / page_rows];
-        if (blk < 0 || blk >= num_blocks) { bad = true; return nullptr; }
-        return tensor_base + (((size_t)blk * Hkv + h) * page_rows + slot % page_rows) * (size_t)chunks;
+        const long long o = rows.at(b, h, slot, Hkv, S_max, chunks);
+        if (o < 0) { bad = true; return nullptr; }
+        return tensor_base + o;
     };
     for (int k0 = 0; k0 < L; k0 += kCompactRows) {
         if (threadIdx.x < kCompactRows) {
@@ -222,7 +233,7 @@ accept_commit_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, cons
                      const int32_t* __restrict__ target, const int32_t* __restrict__ parents,
                      const int32_t* __restrict__ kv_len, int32_t* __restrict__ path, int32_t* __restrict__ accept_len,
                      int32_t* __restrict__ bonus, int32_t* __restrict__ kv_len_out, int N, int Hkv, int D, int S_max,
-                     int* status) {
+                     int* status, const RowMap rows) {
     __shared__ uint4 stage[2][kCompactRows][16];
     __shared__ int32_t par[VISPEC_MAX_TREE_NODES];
     __shared__ int32_t tgt[VISPEC_MAX_TREE_NODES];
@@ -252,35 +263,42 @@ accept_commit_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, cons
     const int tensor = threadIdx.x >> 7;             // 0: K, 1: V
     const int r = (threadIdx.x & 127) >> 3;          // row of the pass, 0..15
     const int c0 = threadIdx.x & 7;                  // this thread moves chunks c0 and c0 + 8
-    uint4* base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]) +
-                  ((size_t)b * Hkv + h) * (size_t)S_max * chunks;
+    uint4* const tensor_base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]);
+    bool bad = false;
     for (int k0 = 0; k0 < L; k0 += kCompactRows) {
         const int k = k0 + r;
         const int s = (k < L && spath[k] != k) ? spath[k] : -1;     // -1: nothing to move
-        if (s >= 0) {
-            const uint4* src = base + (size_t)(S + s) * chunks;
+        const long long so = s >= 0 ? rows.at(b, h, S + s, Hkv, S_max, chunks) : -1;
+        const long long d_off = s >= 0 ? rows.at(b, h, S + k, Hkv, S_max, chunks) : -1;
+        if (s >= 0 && (so < 0 || d_off < 0)) bad = true;               // table entry outside the pool: move dropped
+        const bool move = so >= 0 && d_off >= 0;
+        if (move) {
+            const uint4* src = tensor_base + so;
             if (c0 < chunks) stage[tensor][r][c0] = src[c0];
             if (c0 + 8 < chunks) stage[tensor][r][c0 + 8] = src[c0 + 8];
         }
         __syncthreads();
-        if (s >= 0) {
-            uint4* dst = base + (size_t)(S + k) * chunks;
+        if (move) {
+            uint4* dst = tensor_base + d_off;
             if (c0 < chunks) dst[c0] = stage[tensor][r][c0];
             if (c0 + 8 < chunks) dst[c0 + 8] = stage[tensor][r][c0 + 8];
         }
         __syncthreads();
     }
+    if (bad) record_status(status, VISPEC_E_RANGE);
     if (kv_len_out && writer && threadIdx.x == 0) kv_len_out[b] = S + L;
 }
 
 cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int layer_end, const int32_t* draft,
                                  const int32_t* target, const int32_t* parents, const int32_t* kv_len,
                                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, int B, int N,
-                                 int Hkv, int D, int S_max, int* status, cudaStream_t st) {
+                                 int Hkv, int D, int S_max, int* status, cudaStream_t st, const int32_t* block_table,
+                                 int table_stride, int page_rows, int num_blocks) {
     if (B == 0 || layer_end <= layer_begin) return cudaSuccess;
     dim3 grid(Hkv, B, layer_end - layer_begin);
+    const RowMap rows = {block_table, table_stride, page_rows, num_blocks};
     accept_commit_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, draft, target, parents, kv_len, path,
-                                               accept_len, bonus, kv_len_out, N, Hkv, D, S_max, status);
+                                               accept_len, bonus, kv_len_out, N, Hkv, D, S_max, status, rows);
     return cudaGetLastError();
 }
 
@@ -311,7 +329,7 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
                  const __nv_bfloat16* __restrict__ v_new, const int32_t* __restrict__ positions,
                  const int32_t* __restrict__ kv_len, __nv_bfloat16* __restrict__ k_cache,
                  __nv_bfloat16* __restrict__ v_cache, double log2_theta, int N, int Hq, int Hkv, int D, int S_max,
-                 int* status) {
+                 int* status, const RowMap rmap) {
     __shared__ double cs[64], sn[64];
     // The attention that follows may start its prologue (and stream cache rows below kv_len, which this kernel never
     // writes) while these blocks run; it waits for this grid to finish before it reads q or a tree row.
@@ -337,7 +355,9 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
         const bool is_k = row < Hq + Hkv;
         const int hk = row - Hq - (is_k ? 0 : Hkv);
         src = reinterpret_cast<const uint4*>((is_k ? k_new : v_new) + (((size_t)b * N + i) * Hkv + hk) * D);
-        dst = reinterpret_cast<uint4*>((is_k ? k_cache : v_cache) + (((size_t)b * Hkv + hk) * S_max + S + i) * D);
+        const long long o = rmap.at(b, hk, S + i, Hkv, S_max, D / 8);
+        if (o >= 0) dst = reinterpret_cast<uint4*>(is_k ? k_cache : v_cache) + o;
+        else { src = nullptr; if ((threadIdx.x % tpr) == 0) record_status(status, VISPEC_E_RANGE); }   // entry outside the pool: row dropped
     }
     uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
     if (src) {
@@ -360,8 +380,10 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
 
 cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,
                              const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
-                             int Hkv, int D, int S_max, int* status, cudaStream_t st) {
+                             int Hkv, int D, int S_max, int* status, cudaStream_t st, const int32_t* block_table,
+                             int table_stride, int page_rows, int num_blocks) {
     if (B == 0) return cudaSuccess;
+    const RowMap rmap = {block_table, table_stride, page_rows, num_blocks};
     cudaLaunchConfig_t cfg = {};
     const int rows_per_block = 128 / (D / 16);
     cfg.gridDim = dim3(N, B, (Hq + 2 * Hkv + rows_per_block - 1) / rows_per_block);
@@ -374,7 +396,7 @@ cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, cons
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, rope_rows_kernel, (__nv_bfloat16*)q, (const __nv_bfloat16*)k_new,
                               (const __nv_bfloat16*)v_new, positions, kv_len, (__nv_bfloat16*)k_cache,
-                              (__nv_bfloat16*)v_cache, log2((double)theta), N, Hq, Hkv, D, S_max, status);
+                              (__nv_bfloat16*)v_cache, log2((double)theta), N, Hq, Hkv, D, S_max, status, rmap);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -297,6 +297,58 @@ int vispec_kv_compact_paged(vispec_ctx* c, int layer_begin, int layer_end, const
     return VISPEC_OK;
 }
 
+// the layers [lb, le) are registered, paged, and share one pool geometry; returns VISPEC_OK or the error
+static int paged_range_check(const vispec_ctx* c, int lb, int le, int table_stride) {
+    if (table_stride < 1) return VISPEC_E_SHAPE;
+    for (int l = lb; l < le; ++l) {
+        if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
+        if (!c->page_rows[l]) return VISPEC_E_UNSUPPORTED;
+        if (c->page_rows[l] != c->page_rows[lb] || c->num_blocks[l] != c->num_blocks[lb]) return VISPEC_E_SHAPE;
+    }
+    if (le > lb && (long long)table_stride * c->page_rows[lb] > (1ll << 30)) return VISPEC_E_SHAPE;
+    return VISPEC_OK;
+}
+
+int vispec_accept_commit_paged(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* draft_ids,
+                               const int32_t* target_ids, const int32_t* parents, const int32_t* kv_len,
+                               const int32_t* block_table, int table_stride, int B, int N, int32_t* path,
+                               int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, void* stream) {
+    if (!c || !draft_ids || !target_ids || !parents || !kv_len || !block_table || !path || !accept_len || !bonus)
+        return VISPEC_E_NULL;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
+    if (layer_begin < 0 || layer_end > s.layers || layer_begin >= layer_end) return VISPEC_E_RANGE;
+    if (kv_len_out == kv_len) return VISPEC_E_SHAPE;
+    const int rc = paged_range_check(c, layer_begin, layer_end, table_stride);
+    if (rc != VISPEC_OK) return rc;
+    const int pr = c->page_rows[layer_begin];
+    if (launch_accept_commit(c->d_cache_ptrs, layer_begin, layer_end, draft_ids, target_ids, parents, kv_len, path,
+                             accept_len, bonus, kv_len_out, B, N, s.Hkv, s.D, table_stride * pr, c->d_status,
+                             (cudaStream_t)stream, block_table, table_stride, pr, c->num_blocks[layer_begin]) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
+int vispec_rope_tree_rows_paged(vispec_ctx* c, int layer, void* q, const void* k_new, const void* v_new,
+                                const int32_t* positions, const int32_t* kv_len, const int32_t* block_table,
+                                int table_stride, int B, int N, float theta, void* stream) {
+    if (!c || !q || !k_new || !v_new || !positions || !kv_len || !block_table) return VISPEC_E_NULL;
+    if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return VISPEC_E_ALIGN;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max || !(theta > 1.f)) return VISPEC_E_SHAPE;
+    if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
+    const int rc = paged_range_check(c, layer, layer + 1, table_stride);
+    if (rc != VISPEC_OK) return rc;
+    const int pr = c->page_rows[layer];
+    if (launch_rope_rows(q, k_new, v_new, positions, kv_len, c->h_k[layer], c->h_v[layer], theta, B, N, s.Hq, s.Hkv,
+                         s.D, table_stride * pr, c->d_status, (cudaStream_t)stream, block_table, table_stride, pr,
+                         c->num_blocks[layer]) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
 int vispec_rope_tree_rows(vispec_ctx* c, int layer, void* q, const void* k_new, const void* v_new,
                           const int32_t* positions, const int32_t* kv_len, int B, int N, float theta, void* stream) {
     if (!c || !q || !k_new || !v_new || !positions || !kv_len) return VISPEC_E_NULL;

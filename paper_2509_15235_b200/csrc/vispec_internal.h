@@ -50,11 +50,15 @@ cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int laye
 cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int layer_end, const int32_t* draft,
                                  const int32_t* target, const int32_t* parents, const int32_t* kv_len,
                                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, int B, int N,
-                                 int Hkv, int D, int S_max, int* status, cudaStream_t st);
+                                 int Hkv, int D, int S_max, int* status, cudaStream_t st,
+                                 const int32_t* block_table = nullptr, int table_stride = 0, int page_rows = 0,
+                                 int num_blocks = 0);
 
 cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,
                              const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
-                             int Hkv, int D, int S_max, int* status, cudaStream_t st);
+                             int Hkv, int D, int S_max, int* status, cudaStream_t st,
+                             const int32_t* block_table = nullptr, int table_stride = 0, int page_rows = 0,
+                             int num_blocks = 0);
 
 cudaError_t launch_accept_sampled(const int32_t* draft_ids, const int32_t* parents, const float* p, const float* p_hat,
                                   const float* u_accept, const float* u_bonus, int B, int N, int V, int32_t* path,

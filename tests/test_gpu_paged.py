@@ -173,6 +173,60 @@ def test_paged_commit_matches_the_oracle_on_the_logical_cache():
     ctx.close()
 
 
+def test_paged_accept_commit_and_rope_match_the_oracle():
+    from paper_2509_15235_b200 import binding
+    import gpu_util as gu
+    cfg = synth.get_config("paper_tree")
+    B, N, Hq, Hkv, D, layers, rows, S_max = 3, cfg.N, 8, 2, 128, 2, 32, 512
+    rng = np.random.Generator(np.random.Philox(31))
+    parents = np.stack([synth.draw_tree(N, 3, 8, rng) for _ in range(B)])
+    ids = [synth.draw_ids(parents[b], 1000, 0.7, rng) for b in range(B)]
+    draft = np.stack([d for d, _ in ids]); target = np.stack([t for _, t in ids])
+    kv_len = np.array([100, 0, S_max - N], dtype=np.int32)
+    _, depth, _ = oracle.tree_mask(parents)
+    positions = (kv_len[:, None] + depth).astype(np.int32)
+    ctx = binding.VerifyContext(B, N, Hq, Hkv, D, S_max, layers)
+    state, table = [], None
+    for l in range(layers):
+        k = synth.normal_bf16((B, Hkv, S_max, D), 300 + l); v = synth.normal_bf16((B, Hkv, S_max, D), 310 + l)
+        pools, table = _page((k, v), rows, np.random.Generator(np.random.Philox(32)))
+        kd, vd = gu.bf16_dev(pools[0]), gu.bf16_dev(pools[1])
+        ctx.cache_register_paged(l, kd, vd)
+        state.append([k, v, kd, vd])
+    tab_d = gu.i32_dev(table)
+    # RoPE + placement on every layer, then acceptance + commit over both layers in one launch
+    for l in range(layers):
+        q = synth.normal_bf16((B, N, Hq, D), 320 + l); kn = synth.normal_bf16((B, N, Hkv, D), 330 + l)
+        vn = synth.normal_bf16((B, N, Hkv, D), 340 + l)
+        qd = gu.bf16_dev(q)
+        ctx.rope_tree_rows_paged(l, qd, gu.bf16_dev(kn), gu.bf16_dev(vn), gu.i32_dev(positions), gu.i32_dev(kv_len), tab_d, 1e4)
+        wq, wk, wv, skipped = oracle.rope_rows(q, kn, vn, positions, kv_len, state[l][0], state[l][1], 1e4)
+        assert skipped == 0
+        torch.cuda.synchronize()
+        gk = _unpage(gu.bf16_bits(state[l][2]), table, S_max); gv = _unpage(gu.bf16_bits(state[l][3]), table, S_max)
+        assert np.array_equal(gv, wv)
+        step = np.abs(gk.astype(np.int32) - wk.astype(np.int32))          # bit patterns of equal sign: steps
+        assert step.max() <= 1 and (step != 0).mean() <= 1e-4
+        assert np.abs(gu.bf16_bits(qd).astype(np.int32) - wq.astype(np.int32)).max() <= 1
+        state[l][0], state[l][1] = gk, gv                                  # the commit below starts from what the GPU holds
+    path = torch.zeros((B, N), dtype=torch.int32, device="cuda")
+    alen = torch.zeros(B, dtype=torch.int32, device="cuda"); bonus = torch.zeros(B, dtype=torch.int32, device="cuda")
+    new_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.accept_commit_paged(0, layers, gu.i32_dev(draft), gu.i32_dev(target), gu.i32_dev(parents), gu.i32_dev(kv_len),
+                            tab_d, path, alen, bonus, new_len)
+    torch.cuda.synchronize()
+    assert ctx.status_poll() == 0
+    wp, wl, wb = oracle.accept(draft, target, parents)
+    assert np.array_equal(path.cpu().numpy(), wp) and np.array_equal(alen.cpu().numpy(), wl)
+    assert np.array_equal(bonus.cpu().numpy(), wb) and (wl > 1).any()
+    for l in range(layers):
+        wk, wv, wn = oracle.kv_compact(state[l][0], state[l][1], wp, wl, kv_len)
+        assert np.array_equal(_unpage(gu.bf16_bits(state[l][2]), table, S_max), wk)
+        assert np.array_equal(_unpage(gu.bf16_bits(state[l][3]), table, S_max), wv)
+        assert np.array_equal(new_len.cpu().numpy(), wn)
+    ctx.close()
+
+
 def test_paged_host_errors():
     from paper_2509_15235_b200 import binding
     ctx = binding.VerifyContext(2, 8, 4, 2, 128, 256, 2)
