@@ -106,8 +106,12 @@ typedef enum vispec_option {
     VISPEC_OPT_FORCE_GENERIC = 2,
     /* Default 0.  How the TMA/tcgen05 attention kernel combines the pieces of a (sequence, kv head) that
      * several thread blocks work on: 0 chooses per call; 1 always parks partial results in the workspace
-     * and merges them with a second kernel; 2 uses thread-block clusters that merge through distributed
-     * shared memory whenever the shape allows one cluster per (sequence, kv head, row block). */
+     * (they are merged by the block that delivers a unit's last partial when a unit has at most 64 query rows,
+     * by a second kernel otherwise); 2 uses thread-block clusters that merge through distributed shared memory
+     * whenever the shape allows one cluster per (sequence, kv head, row block); 3 is 1 with the second kernel
+     * always.  The in-kernel merge counts arrivals in the first 64 KiB of the workspace, which
+     * vispec_ctx_set_workspace zeroes and every call leaves zero (a call that ended with VISPEC_E_TIMEOUT may
+     * not: set the workspace again after one). */
     VISPEC_OPT_SPLIT_FORM = 3
 } vispec_option;
 

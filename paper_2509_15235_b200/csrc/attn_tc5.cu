@@ -85,7 +85,7 @@ constexpr long long kWaitCycles = 1500000000LL;                // ~0.8 s at 1.9 
 enum { B_KFULL = 0, B_KEMPTY = B_KFULL + NSK, B_VFULL = B_KEMPTY + NSK, B_VEMPTY = B_VFULL + NSV,
        B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2,
        B_QFULL = B_PVDONE + 2, B_PAIRX = B_QFULL + 1, B_XCH = B_PAIRX + 4, B_XFREE = B_XCH + 1,
-       B_COUNT = B_XFREE + 1 };
+       B_SEGSYNC = B_XFREE + 1, B_COUNT = B_SEGSYNC + 1 };
 static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block too small");
 
 // The schedule every CTA (and the merge kernel) derives from kv_len.
@@ -391,6 +391,82 @@ struct SegIter {
     }
 };
 
+// One (row, 16 output columns) of a unit: the partials of CTAs c0..c1 (slot 2c if the unit starts CTA c's range,
+// else 2c + 1) folded into the final output.  Shared by the merge kernel and by the attention kernel's own merge.
+template <int ROWS>
+__device__ __forceinline__ void merge_row_cols(const float4* __restrict__ part_o, const float2* __restrict__ part_ml,
+                                               __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int T, int geff,
+                                               int ub, int c0, int c1, int b, int node, int head, int Hq, int N,
+                                               int lrow, int cw) {
+    auto slot_of = [&](int c) { return cta_lo(c, T, geff) >= ub ? 2 * c : 2 * c + 1; };
+    // Segments are taken four at a time with every load of a group issued before the first use, so that a
+    // group costs one memory round trip; groups are folded with the usual running-maximum rescale.
+    float m_all = -INFINITY, l_all = 0.f;
+    float4 acc[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int cb = c0; cb <= c1; cb += 4) {
+        float2 ml[4];
+        float4 v[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = cb + j;
+            ml[j] = make_float2(-INFINITY, 0.f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v[j][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c <= c1) {
+                const int slot = slot_of(c);
+                ml[j] = __ldcg(&part_ml[(size_t)slot * ROWS + lrow]);
+                const float4* src = part_o + ((size_t)slot * 32 + cw * 4) * ROWS + lrow;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) v[j][k] = __ldcg(src + (size_t)k * ROWS);
+            }
+        }
+        float m_new = m_all;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m_new = fmaxf(m_new, ml[j].x);
+        const float m_fin = (m_new == -INFINITY) ? 0.f : m_new;
+        const float a = exp2f(m_all - m_fin);                 // 0 while nothing has been accumulated
+        l_all *= a;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { acc[k].x *= a; acc[k].y *= a; acc[k].z *= a; acc[k].w *= a; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float w = exp2f(ml[j].x - m_fin);           // 0 for a segment that saw nothing (or is absent)
+            l_all += ml[j].y * w;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc[k].x += w * v[j][k].x; acc[k].y += w * v[j][k].y; acc[k].z += w * v[j][k].z; acc[k].w += w * v[j][k].w;
+            }
+        }
+        m_all = m_new;
+    }
+    const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+    __nv_bfloat16* orow = out + (((size_t)b * N + node) * Hq + head) * D + cw * 16;
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+        *reinterpret_cast<uint4*>(orow + k * 8) =
+            make_uint4(pack_bf16(acc[2 * k].x * inv, acc[2 * k].y * inv), pack_bf16(acc[2 * k].z * inv, acc[2 * k].w * inv),
+                       pack_bf16(acc[2 * k + 1].x * inv, acc[2 * k + 1].y * inv), pack_bf16(acc[2 * k + 1].z * inv, acc[2 * k + 1].w * inv));
+    if (lse && cw == 0)
+        lse[((size_t)b * Hq + head) * N + node] = l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+}
+
+// The whole unit, by the 256 softmax threads of the CTA that delivered the unit's last partial (thread st of 256).
+// Not inlined: its accumulators stay out of the attention kernel's register budget.
+struct MergeArgs { const float4* part_o; const float2* part_ml; __nv_bfloat16* out; float* lse; int Hq, G, N, rows_total; };
+template <int ROWS>
+__device__ __noinline__ void merge_unit(const MergeArgs m, int T, int geff, int ub, int c0, int c1, int b, int kvh,
+                                        int mblock, int st) {
+    for (int item = st; item < ROWS * 8; item += kSmx) {
+        const int cw = item / ROWS, lrow = item - cw * ROWS;
+        const int row = mblock * 128 + lrow;
+        if (row >= m.rows_total) continue;
+        merge_row_cols<ROWS>(m.part_o, m.part_ml, m.out, m.lse, T, geff, ub, c0, c1, b, row / m.G, kvh * m.G + row % m.G,
+                             m.Hq, m.N, lrow, cw);
+    }
+}
+
 // ---- producer of a paged segment ---------------------------------------------------------------------
 // Paged cache: a step's 128 slots are 128 / page_rows pool blocks, each its own box.  Run by the whole producer
 // warp: lane j owns block j of every step - its table entry and its four copies (two d-halves of K and of V) -
@@ -404,7 +480,8 @@ struct SegIter {
 // step << 28 | a wait gave up << 29 | has waited for the preceding kernel << 30 (the same in every lane).
 constexpr int kTabRing = 8, kTabAhead = 6;     // steps held in the ring / steps a copy is issued ahead
 // pool [num_blocks][Hkv][page_rows][D]; block_table[b][i] = pool block of logical slots [i * page_rows, (i + 1) * page_rows)
-struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N; int* status; };
+struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N; int* status;
+                   int* unit_counters; };   // even split: arrivals per unit (all zero between calls); nullptr: a merge kernel follows
 __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensorMap* k_map, const CUtensorMap* v_map,
                                                int b, int kvh, int st0, int n, int S, uint32_t base, uint32_t bars,
                                                uint32_t ring, volatile int* abort_flag, uint64_t pol, int it,
@@ -486,6 +563,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     const uint32_t bars = base + SMEM_BAR;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + SMEM_BAR + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SMEM_BAR + B_COUNT * 8 + 8);
+    volatile int* seg_flag = abort_flag + 1;               // this CTA delivered the last partial of the unit just finished
     Sched& sched = *reinterpret_cast<Sched*>(sm + SMEM_SCHED);
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
@@ -504,6 +582,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         for (int i = 0; i < 4; ++i) mbar_init(bar(B_PAIRX + i), 64);
         mbar_init(bar(B_QFULL), kSmx);
         mbar_init(bar(B_XCH), 128); mbar_init(bar(B_XFREE), 128);
+        mbar_init(bar(B_SEGSYNC), kSmx);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -668,6 +747,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         float* xm = reinterpret_cast<float*>(sm + SMEM_XM);   // [2 step parities][2 column halves][128 lanes] tile maxima;
                                                               // in the epilogue: [0..255] l by (ch, lane), [256..383] m by lane
         int px = 0;                                           // phases of the pair barrier used so far
+        int sx = 0;                                           // phases of the segment barrier used so far
         pdl_wait();                                           // q, tree_mask and every output come after the preceding kernel
         if (tid == 128) { TL_START(p.trace_idx, 2); TL_END(p.trace_idx, 3); }
         CTA_TS(2);
@@ -980,6 +1060,32 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     }
                     if (PAIR) mbar_arrive(bar(B_XFREE));
                 }
+                if (PAIR && !CL && pa.unit_counters && sg.slot >= 0) {
+                    // ---- even split without a merge kernel (rows <= 64 only: with 128 rows the merge kernel is faster): the CTA that delivers a unit's last partial merges the
+                    // unit.  Nobody waits for another CTA: a fence, one atomic per segment, and the last arrival
+                    // reads the others' partials (written before their fences) from L2. ----
+                    __threadfence();
+                    mbar_arrive(bar(B_SEGSYNC));                       // every softmax thread has written and fenced
+                    if (!mbar_wait_warp(bar(B_SEGSYNC), sx & 1, abort_flag)) { ok = false; break; }
+                    ++sx;
+                    const int uib = sg.kvh * p.n_mblocks + sg.mblock;
+                    const int ub = sched.base[sg.b] + uib * sg.steps;
+                    const int c0 = cta_of(ub, T, geff), c1 = cta_of(ub + sg.steps - 1, T, geff);
+                    if (st == 0) {
+                        int* cnt = pa.unit_counters + (sg.b * p.Hkv * p.n_mblocks + uib);
+                        const bool last = atomicAdd(cnt, 1) == c1 - c0;
+                        if (last) *cnt = 0;                            // all zero again for the next call
+                        *seg_flag = last ? 1 : 0;
+                    }
+                    mbar_arrive(bar(B_SEGSYNC));
+                    if (!mbar_wait_warp(bar(B_SEGSYNC), sx & 1, abort_flag)) { ok = false; break; }
+                    ++sx;
+                    if (*seg_flag) {
+                        __threadfence();
+                        const MergeArgs ma = {p.part_o, p.part_ml, p.out, p.lse, p.Hq, G, N, rows_total};
+                        merge_unit<ROWS>(ma, T, geff, ub, c0, c1, sg.b, sg.kvh, sg.mblock, st);
+                    }
+                }
                 if (CL) TRACE_MISC(12);
                 tc_fence_before();        // the next segment's first product overwrites O
                 TRACE_MISC(7);
@@ -1107,58 +1213,7 @@ attn_tc5_merge_kernel(const Tc5Params p) {
     if (row >= G * N) { TL_END(p.trace_idx, 2); return; }
     const int node = row / G, head = kvh * G + row % G;
 
-    auto slot_of = [&](int c) { return cta_lo(c, T, geff) >= ub ? 2 * c : 2 * c + 1; };
-    // Segments are taken four at a time with every load of a group issued before the first use, so that a
-    // group costs one memory round trip; groups are folded with the usual running-maximum rescale.
-    float m_all = -INFINITY, l_all = 0.f;
-    float4 acc[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int cb = c0; cb <= c1; cb += 4) {
-        float2 ml[4];
-        float4 v[4][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int c = cb + j;
-            ml[j] = make_float2(-INFINITY, 0.f);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) v[j][k] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c <= c1) {
-                const int slot = slot_of(c);
-                ml[j] = __ldcg(&p.part_ml[(size_t)slot * ROWS + lrow]);
-                const float4* src = p.part_o + ((size_t)slot * 32 + cw * 4) * ROWS + lrow;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) v[j][k] = __ldcg(src + (size_t)k * ROWS);
-            }
-        }
-        float m_new = m_all;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) m_new = fmaxf(m_new, ml[j].x);
-        const float m_fin = (m_new == -INFINITY) ? 0.f : m_new;
-        const float a = exp2f(m_all - m_fin);                 // 0 while nothing has been accumulated
-        l_all *= a;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) { acc[k].x *= a; acc[k].y *= a; acc[k].z *= a; acc[k].w *= a; }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float w = exp2f(ml[j].x - m_fin);           // 0 for a segment that saw nothing (or is absent)
-            l_all += ml[j].y * w;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                acc[k].x += w * v[j][k].x; acc[k].y += w * v[j][k].y; acc[k].z += w * v[j][k].z; acc[k].w += w * v[j][k].w;
-            }
-        }
-        m_all = m_new;
-    }
-    const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
-    __nv_bfloat16* orow = p.out + (((size_t)b * N + node) * p.Hq + head) * D + cw * 16;
-#pragma unroll
-    for (int k = 0; k < 2; ++k)
-        *reinterpret_cast<uint4*>(orow + k * 8) =
-            make_uint4(pack_bf16(acc[2 * k].x * inv, acc[2 * k].y * inv), pack_bf16(acc[2 * k].z * inv, acc[2 * k].w * inv),
-                       pack_bf16(acc[2 * k + 1].x * inv, acc[2 * k + 1].y * inv), pack_bf16(acc[2 * k + 1].z * inv, acc[2 * k + 1].w * inv));
-    if (p.lse && cw == 0)
-        p.lse[((size_t)b * p.Hq + head) * N + node] = l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+    merge_row_cols<ROWS>(p.part_o, p.part_ml, p.out, p.lse, T, geff, ub, c0, c1, b, node, head, p.Hq, N, lrow, cw);
     TL_END(p.trace_idx, 2);
 }
 
@@ -1375,7 +1430,12 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
 #endif
     cudaError_t err;
     const bool paged = a.page_rows != 0;
-    const PagedArgs pa = {a.block_table, a.table_stride, a.page_rows, a.num_blocks, a.Hkv, a.N, a.status};
+    // even split, at most 64 rows per unit: the arrival counters at the head of the workspace serve the in-kernel
+    // merge (measured: 68.8 against 70.3 us per layer on llava13b_b4; with 128 rows it lost, 65.9 against 60.5 us on
+    // qwen3b_S32768_N16_B8, so those, a grid with more units than counters, and split form 3 get the merge kernel)
+    const bool own_merge = pair && ck == 0 && a.tc5_path != 3 && (size_t)units * sizeof(int) <= kCounterBytes;
+    const PagedArgs pa = {a.block_table, a.table_stride, a.page_rows, a.num_blocks, a.Hkv, a.N, a.status,
+                          own_merge ? (int*)a.ws : nullptr};
     auto launch_attn = [&](auto kernel, int cluster) {
         return launch_pdl(kernel, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, cluster, *a.k_map, *a.v_map, p, pa);
     };
@@ -1391,6 +1451,7 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
                 : (pair ? launch_attn(attn_tc5_kernel<true, false, false>, 0) : launch_attn(attn_tc5_kernel<false, false, false>, 0));
     if (err != cudaSuccess) return err;
     ++*n_launches;
+    if (own_merge) return cudaSuccess;
     err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p)
                : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 8), dim3(128), 0, st, 0, p);
     if (err != cudaSuccess) return err;

@@ -129,7 +129,7 @@ int vispec_ctx_set_option(vispec_ctx* c, int option, int value) {
         case VISPEC_OPT_EARLY_PREFETCH: c->early_prefetch = value != 0; return VISPEC_OK;
         case VISPEC_OPT_FORCE_GENERIC: c->force_generic = value != 0; return VISPEC_OK;
         case VISPEC_OPT_SPLIT_FORM:
-            if (value < 0 || value > 2) return VISPEC_E_RANGE;
+            if (value < 0 || value > 3) return VISPEC_E_RANGE;
             c->tc5_path = value; return VISPEC_OK;
         default: return VISPEC_E_UNSUPPORTED;
     }

@@ -58,7 +58,7 @@ def test_tiny_config_full_parity(gu):
     (4, 2, 128, 31, 1000, 1088),  # the paper's 30-token tree plus root
     (3, 3, 128, 65, 130, 256),    # two mask words
 ])
-@pytest.mark.parametrize("split_form", [0, 1, 2])
+@pytest.mark.parametrize("split_form", [0, 1, 2, 3])
 def test_shapes_span_tiles_tails_and_group_sizes(gu, Hq, Hkv, D, N, S, S_max, split_form):
     rng = np.random.Generator(np.random.Philox(Hq * 1000 + N))
     B = 2

@@ -72,7 +72,7 @@ def _case(B, N, Hq, Hkv, S_list, S_max, seed):
 
 
 @pytest.mark.parametrize("page_rows", [16, 32, 64, 128])
-@pytest.mark.parametrize("split_form", [0, 1, 2])
+@pytest.mark.parametrize("split_form", [0, 1, 2, 3])
 def test_paged_attention_equals_contiguous_and_oracle(page_rows, split_form):
     import gpu_util as gu
     B, N, Hq, Hkv, S_max = 3, 60, 8, 2, 1152
