@@ -1359,18 +1359,27 @@ static int query_max_clusters(bool pair, int k) {
 // Cluster size for the cluster form, or 0 when the even split with partials in global memory serves better:
 // one cluster per unit, all clusters co-resident, and three quarters of the SMs in use (three fifths for short calls).
 static int tc5_cluster_size(const AttnArgs& a, int units) {
-    if (a.tc5_path == 1) return 0;
-    const bool pair = (a.Hq / a.Hkv) * a.N <= 64;
+    if (a.tc5_path == 1 || a.tc5_path == 3) return 0;
+    const int rows_total = (a.Hq / a.Hkv) * a.N;
+    const bool pair = rows_total <= 64;
     int best = 0;
     for (int k = 1; k <= 8; ++k)
         if (units * k <= a.sm_count && g_max_clusters[pair][k] >= units) best = k;
     if (best == 0) return 0;
     if (a.tc5_path == 2) return best;
-    if (units * best * 4 >= a.sm_count * 3) return best;
-    // Fewer CTAs than that pay off only for short calls, where the second launch and the partials of the even
-    // split weigh more than the idle SMs: at most 8 steps per CTA if every SM were used.
-    const long long t_max = (long long)units * ((a.S_max + STEP - 1) / STEP);
-    return (units * best * 5 >= a.sm_count * 3 && t_max <= 8ll * a.sm_count) ? best : 0;
+    // Both forms, estimated in microseconds from what was measured over the workloads (the long-response sweep
+    // cells, the 7B and 13B shapes): a fixed part (11 for the cluster form, 14 for the even split with its partials
+    // and second phase), the steps of the busiest CTA at 1.2 per step or at the HBM share of that many CTAs (64 KB
+    // per step at 5.2 TB/s over the cluster form's CTAs, 6.6 TB/s over the even split's; the row blocks of one kv
+    // head read the same tiles, so only one in n_mblocks comes from HBM), and 0.25 per partial a unit is merged
+    // from.  The host knows only the capacity S_max, not kv_len: the estimate is for full caches.
+    const int n_mblocks = pair ? 1 : (rows_total + 127) / 128;
+    const double steps = (double)((a.S_max + STEP - 1) / STEP), T = steps * units;
+    const double n_c = (double)units * best, per_c = (double)(((a.S_max + STEP - 1) / STEP + best - 1) / best);
+    const double est_c = 11.0 + per_c * fmax(1.2, n_c * 0.0125 / n_mblocks);
+    const double n_e = fmin((double)a.sm_count, fmax(1.0, T / 2.0));
+    const double est_e = 14.0 + (T / n_e) * fmax(1.2, n_e * 0.00973 / n_mblocks) + 0.25 * (n_e / units);
+    return est_c <= est_e ? best : 0;
 }
 
 bool attn_tc5_supports(const AttnArgs& a) {
