@@ -1,6 +1,6 @@
 """Pins of the sampled-acceptance oracle (CPU only), against what the paper and the mathematics fix:
 
-* hand-worked two-round example (tests/golden/sampled_two_rounds.json): the thresholds of the uniforms at which
+* hand-worked two-sibling example (tests/golden/sampled_two_siblings.json): the thresholds of the uniforms at which
   the decisions flip, and the bonus token once both siblings are rejected;
 * p = p^: every first child is kept (ratio 1), so the path is the first-child chain;
 * one-hot draft distribution: keep probability is p(x), the residual is p with x removed;
@@ -16,7 +16,7 @@ import numpy as np
 
 import oracle
 
-GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "sampled_two_rounds.json")
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "sampled_two_siblings.json")
 
 
 def _one(draft_ids, parents, p_rows, ph_rows, ua, ub):
@@ -26,7 +26,7 @@ def _one(draft_ids, parents, p_rows, ph_rows, ua, ub):
     return list(path[0][:alen[0]]), int(bonus[0])
 
 
-def test_hand_worked_two_round_thresholds():
+def test_hand_worked_two_sibling_thresholds():
     g = json.load(open(GOLDEN))
     ph = [g["p_hat"]] * 3
     for case in g["cases"]:
