@@ -58,6 +58,7 @@ def parse_args():
     ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context: 0 automatic, 1 partials + merge kernel, 2 clusters")
     ap.add_argument("--no-sampled", action="store_true", help="skip the timing of vispec_accept_sampled")
     ap.add_argument("--paged", type=int, default=0, help="serve the caches from a block pool of this many slots per block (16/32/64/128)")
+    ap.add_argument("--token-major", action="store_true", help="with --paged: pool blocks are [slots, kv heads, D] instead of [kv heads, slots, D]")
     ap.add_argument("--with-rope", action="store_true", help="also run vispec_rope_tree_rows before each layer's attention")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying graphs")
     return ap.parse_args()
@@ -205,7 +206,7 @@ class DeviceWorkload:
         self.theta = theta
         self.with_rope = True
 
-    def enable_paging(self, page_rows):
+    def enable_paging(self, page_rows, token_major=False):
         """Re-home every layer's cache in a block pool [num_blocks, Hkv, page_rows, D] with the blocks in a seeded
         random order (what a serving stack's allocator leaves behind) and serve the step through the *_paged calls."""
         torch, cfg = self.torch, self.cfg
@@ -220,9 +221,9 @@ class DeviceWorkload:
                 blocks = c.view(B, Hkv, per, page_rows, D).permute(0, 2, 1, 3, 4).reshape(B * per, Hkv, page_rows, D)
                 pool = torch.empty(blocks.shape, dtype=blocks.dtype, device=blocks.device)
                 pool[perm] = blocks
-                pools.append(pool)
+                pools.append(pool.permute(0, 2, 1, 3).contiguous() if token_major else pool)
             self.k[l], self.v[l] = pools
-            self.ctx.cache_register_paged(l, self.k[l], self.v[l])
+            self.ctx.cache_register_paged(l, self.k[l], self.v[l], token_major)
         self.page_rows = page_rows
 
     def _pre(self):
@@ -419,7 +420,7 @@ def main():
         wl.ctx.ctx_set_option(binding.OPT_SPLIT_FORM, args.split_form)
     L = wl.L
     if args.paged:
-        wl.enable_paging(args.paged)
+        wl.enable_paging(args.paged, args.token_major)
     if args.with_rope:
         wl.enable_rope(tree, 1e6 if cfg.name.startswith("qwen") else 1e4)
 
@@ -576,7 +577,7 @@ def main():
                    "kv_bytes_per_layer": wl.kv_bytes_per_layer,
                    "l2": f"inputs larger than L2: {L} layers x {wl.kv_bytes_per_layer / 1e6:.1f} MB rotate, no flush",
                    "launch": "plain C-ABI calls" if args.no_graph else "C-ABI calls captured once, replayed as 3 CUDA graphs per step",
-                   "rope_tree_rows": bool(args.with_rope), "paged_block_rows": args.paged,
+                   "rope_tree_rows": bool(args.with_rope), "paged_block_rows": args.paged, "paged_token_major": bool(args.token_major),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
         "attn_us_per_layer": attn_s * 1e6,

@@ -184,12 +184,14 @@ int vispec_tree_verify_attn_static(const void* q, const void* k_cache, const voi
 
 /* Paged cache (the paper's runtime uses one pre-allocated cache per sequence, App. A; a serving stack shares a
  * pool of fixed-size blocks between sequences instead - same arithmetic, another layout).
- *   k_pool, v_pool: bf16 [num_blocks, Hkv, page_rows, D] (device, 128-byte aligned, caller-owned), page_rows in
- *   {16, 32, 64, 128}, D = 128 only (E_UNSUPPORTED otherwise).  Registering a layer replaces what was registered
+ *   k_pool, v_pool: bf16 [num_blocks, Hkv, page_rows, D], or [num_blocks, page_rows, Hkv, D] if token_major != 0
+ *   (device, 128-byte aligned, caller-owned), page_rows in {16, 32, 64, 128}, D = 128 only (E_UNSUPPORTED
+ *   otherwise).  Registering a layer replaces what was registered
  *   for it before, paged or not.  A paged layer is served by the *_paged calls only (the others answer
  *   E_UNSUPPORTED for it, and the *_paged calls answer E_UNSUPPORTED for a contiguous layer).
  * Host errors: E_NULL, E_RANGE (layer), E_ALIGN, E_UNSUPPORTED, E_SHAPE. */
-int vispec_cache_register_paged(vispec_ctx* ctx, int layer, void* k_pool, void* v_pool, int num_blocks, int page_rows);
+int vispec_cache_register_paged(vispec_ctx* ctx, int layer, void* k_pool, void* v_pool, int num_blocks, int page_rows,
+                                int token_major);
 
 /* vispec_tree_verify_attn on a paged layer.  block_table [B, table_stride] int32 (device): entry i of row b is
  * the pool block that holds logical slots [i * page_rows, (i + 1) * page_rows) of sequence b; only the entries of
@@ -207,7 +209,7 @@ int vispec_tree_verify_attn_paged(vispec_ctx* ctx, int layer, const void* q, con
 
 /* vispec_kv_compact on paged layers [layer_begin, layer_end): rows move between logical slots kv_len + path[k]
  * and kv_len + k, each found through block_table (one table serves all layers of the range, which must share
- * num_blocks and page_rows: E_SHAPE otherwise).  A table entry outside the pool drops that row's move and sets
+ * num_blocks, page_rows and layout: E_SHAPE otherwise).  A table entry outside the pool drops that row's move and sets
  * the status word VISPEC_E_RANGE.  Other arguments and errors as in vispec_kv_compact. */
 int vispec_kv_compact_paged(vispec_ctx* ctx, int layer_begin, int layer_end, const int32_t* path,
                             const int32_t* accept_len, const int32_t* kv_len, const int32_t* block_table,

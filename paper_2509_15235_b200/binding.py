@@ -73,7 +73,7 @@ def load() -> ctypes.CDLL:
             "vispec_stream_probe": [vp, ci, vp, ci, ci, vp],
             "vispec_accept_sampled": [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp],
             "vispec_tree_rerank": [vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp],
-            "vispec_cache_register_paged": [vp, ci, vp, vp, ci, ci],
+            "vispec_cache_register_paged": [vp, ci, vp, vp, ci, ci, ci],
             "vispec_tree_verify_attn_paged": [vp, ci, vp, vp, vp, ci, vp, ci, ci, cf, vp, vp, vp],
             "vispec_kv_compact_paged": [vp, ci, ci, vp, vp, vp, vp, ci, vp, ci, ci, vp],
             "vispec_accept_commit_paged": [vp, ci, ci, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, vp, vp],
@@ -220,10 +220,12 @@ class VerifyContext:
                                            _ptr(parents), _ptr(draft_ids), _ptr(selected), _stream()),
                "vispec_tree_rerank")
 
-    def cache_register_paged(self, layer: int, k_pool: torch.Tensor, v_pool: torch.Tensor) -> None:
-        num_blocks, _, page_rows, _ = k_pool.shape
-        _check(self.lib.vispec_cache_register_paged(self.handle, layer, _ptr(k_pool), _ptr(v_pool), num_blocks, page_rows),
-               "vispec_cache_register_paged")
+    def cache_register_paged(self, layer: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
+                             token_major: bool = False) -> None:
+        """Pools [num_blocks, Hkv, page_rows, D], or [num_blocks, page_rows, Hkv, D] with token_major."""
+        num_blocks, page_rows = k_pool.shape[0], k_pool.shape[1 if token_major else 2]
+        _check(self.lib.vispec_cache_register_paged(self.handle, layer, _ptr(k_pool), _ptr(v_pool), num_blocks, page_rows,
+                                                    int(token_major)), "vispec_cache_register_paged")
         self._caches[layer] = (k_pool, v_pool)   # keep the tensors alive
 
     def tree_verify_attn_paged(self, layer: int, q: torch.Tensor, kv_len: torch.Tensor, block_table: torch.Tensor,

@@ -479,8 +479,10 @@ __device__ __noinline__ void merge_unit(const MergeArgs m, int T, int geff, int 
 // everything by value, so that the caller's counters stay in registers.  Returns steps issued in full | K-only
 // step << 28 | a wait gave up << 29 | has waited for the preceding kernel << 30 (the same in every lane).
 constexpr int kTabRing = 8, kTabAhead = 6;     // steps held in the ring / steps a copy is issued ahead
-// pool [num_blocks][Hkv][page_rows][D]; block_table[b][i] = pool block of logical slots [i * page_rows, (i + 1) * page_rows)
-struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N; int* status;
+// pool [num_blocks][Hkv][page_rows][D] (tensor map (d, slot, block * Hkv + head)) or, token_major,
+// [num_blocks][page_rows][Hkv][D] (tensor map (d, head, block * page_rows + slot));
+// block_table[b][i] = pool block of logical slots [i * page_rows, (i + 1) * page_rows)
+struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N, token_major; int* status;
                    int* unit_counters; };   // even split: arrivals per unit (all zero between calls); nullptr: a merge kernel follows
 __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensorMap* k_map, const CUtensorMap* v_map,
                                                int b, int kvh, int st0, int n, int S, uint32_t base, uint32_t bars,
@@ -507,12 +509,16 @@ __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensor
         const int tok = (st0 + t) * STEP;
         if (!waited && tok + STEP > S) { pdl_wait(); waited = true; }   // the tree's rows come from the preceding kernel
         const bool load = mine && tok + lane * p.page_rows < total;
-        int z = -1;                                                      // -1: out of the pool, reads as zeros
+        int c1 = 0, c2 = -p.page_rows;                                   // a box outside the pool: reads as zeros
         if (load) {
             int e;
             asm volatile("ld.shared.s32 %0, [%1];" : "=r"(e) : "r"(ring + 4u * (uint32_t)((t % kTabRing) * 8 + lane)) : "memory");
-            if (e >= 0 && e < p.num_blocks) z = e * p.Hkv + kvh;
-            else if (p.status) atomicCAS(p.status, 0, VISPEC_E_RANGE);
+            if (e >= 0 && e < p.num_blocks) {
+                c1 = p.token_major ? kvh : 0;
+                c2 = p.token_major ? e * p.page_rows : e * p.Hkv + kvh;
+            } else if (p.status) {
+                atomicCAS(p.status, 0, VISPEC_E_RANGE);
+            }
         }
         const uint32_t tx = (uint32_t)__popc(__ballot_sync(0xffffffffu, load)) * sub_bytes * 2u;
         const int sk = it % NSK, sv = it % NSV;
@@ -524,8 +530,8 @@ __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensor
         w = __shfl_sync(0xffffffffu, w, 0);                              // the byte count is posted before any lane copies
         if (!w) { fail = 2u << 28; break; }
         if (load) {
-            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 0, 0, z, pol);
-            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 64, 0, z, pol);
+            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 0, c1, c2, pol);
+            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 64, c1, c2, pol);
         }
         if (lane == 0) {
             w = mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag);
@@ -534,8 +540,8 @@ __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensor
         w = __shfl_sync(0xffffffffu, w, 0);
         if (!w) { fail = 3u << 28; break; }
         if (load) {
-            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 0, 0, z, pol);
-            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 64, 0, z, pol);
+            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 0, c1, c2, pol);
+            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 64, c1, c2, pol);
         }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");                     // nothing of this segment stays in flight
@@ -1443,7 +1449,7 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     // merge (measured: 68.8 against 70.3 us per layer on llava13b_b4; with 128 rows it lost, 65.9 against 60.5 us on
     // qwen3b_S32768_N16_B8, so those, a grid with more units than counters, and split form 3 get the merge kernel)
     const bool own_merge = pair && ck == 0 && a.tc5_path != 3 && (size_t)units * sizeof(int) <= kCounterBytes;
-    const PagedArgs pa = {a.block_table, a.table_stride, a.page_rows, a.num_blocks, a.Hkv, a.N, a.status,
+    const PagedArgs pa = {a.block_table, a.table_stride, a.page_rows, a.num_blocks, a.Hkv, a.N, a.token_major, a.status,
                           own_merge ? (int*)a.ws : nullptr};
     auto launch_attn = [&](auto kernel, int cluster) {
         return launch_pdl(kernel, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, cluster, *a.k_map, *a.v_map, p, pa);

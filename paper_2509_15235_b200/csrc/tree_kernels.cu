@@ -143,14 +143,15 @@ cudaError_t launch_accept(const int32_t* draft, const int32_t* target, const int
 constexpr int kCompactRows = 16;
 
 // Where logical slot `slot` of (sequence b, kv head h) lives, in 16-byte vectors from the tensor's base.
-// Contiguous cache [B,Hkv,S_max,D]: table == nullptr.  Paged pool [num_blocks,Hkv,page_rows,D]: through the block
-// table; -1 if the table entry is outside the pool.
+// Contiguous cache [B,Hkv,S_max,D]: table == nullptr.  Paged pool [num_blocks,Hkv,page_rows,D], or
+// [num_blocks,page_rows,Hkv,D] if token_major: through the block table; -1 if the table entry is outside the pool.
 struct RowMap {
-    const int32_t* table; int table_stride, page_rows, num_blocks;
+    const int32_t* table; int table_stride, page_rows, num_blocks, token_major;
     __device__ __forceinline__ long long at(int b, int h, int slot, int Hkv, int S_max, int chunks) const {
         if (!table) return (((long long)b * Hkv + h) * S_max + slot) * chunks;
         const int blk = table[(size_t)b * table_stride + slot / page_rows];
         if (blk < 0 || blk >= num_blocks) return -1;
+        if (token_major) return (((long long)blk * page_rows + slot % page_rows) * Hkv + h) * chunks;
         return (((long long)blk * Hkv + h) * page_rows + slot % page_rows) * chunks;
     }
 };
@@ -159,7 +160,8 @@ __global__ void __launch_bounds__(256)
 kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const int32_t* __restrict__ path,
                   const int32_t* __restrict__ accept_len, const int32_t* __restrict__ kv_len,
                   int32_t* __restrict__ kv_len_out, int N, int Hkv, int D, int S_max, int* status,
-                  const int32_t* __restrict__ block_table, int table_stride, int page_rows, int num_blocks) {
+                  const int32_t* __restrict__ block_table, int table_stride, int page_rows, int num_blocks,
+                  int token_major) {
     __shared__ uint4 stage[2][kCompactRows][16];   // up to 256 B per row (D = 128)
     __shared__ int32_t src_row[kCompactRows];
     const int layer = layer_begin + blockIdx.z, b = blockIdx.y, h = blockIdx.x;
@@ -175,7 +177,7 @@ kv_compact_kernel(void* const* __restrict__ cache_ptrs, int layer_begin, const i
     const int c0 = threadIdx.x & 7;                  // this thread moves chunks c0 and c0 + 8
     uint4* const tensor_base = reinterpret_cast<uint4*>(cache_ptrs[2 * layer + tensor]);
     bool bad = false;
-    const RowMap rows = {block_table, table_stride, page_rows, num_blocks};
+    const RowMap rows = {block_table, table_stride, page_rows, num_blocks, token_major};
     // a table entry outside the pool drops the move and is reported
     auto row_of = [&](int slot) -> uint4* {
         const long long o = rows.at(b, h, slot, Hkv, S_max, chunks);
@@ -213,11 +215,12 @@ cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int laye
                               const int32_t* path, const int32_t* accept_len, const int32_t* kv_len,
                               int32_t* kv_len_out, int B, int N, int Hkv, int D, int S_max, int* status,
                               cudaStream_t st, const int32_t* block_table, int table_stride, int page_rows,
-                              int num_blocks) {
+                              int num_blocks, int token_major) {
     if (B == 0 || layer_end <= layer_begin) return cudaSuccess;
     dim3 grid(Hkv, B, layer_end - layer_begin);
     kv_compact_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, path, accept_len, kv_len, kv_len_out,
-                                            N, Hkv, D, S_max, status, block_table, table_stride, page_rows, num_blocks);
+                                            N, Hkv, D, S_max, status, block_table, table_stride, page_rows, num_blocks,
+                                            token_major);
     return cudaGetLastError();
 }
 
@@ -293,10 +296,10 @@ cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int l
                                  const int32_t* target, const int32_t* parents, const int32_t* kv_len,
                                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, int B, int N,
                                  int Hkv, int D, int S_max, int* status, cudaStream_t st, const int32_t* block_table,
-                                 int table_stride, int page_rows, int num_blocks) {
+                                 int table_stride, int page_rows, int num_blocks, int token_major) {
     if (B == 0 || layer_end <= layer_begin) return cudaSuccess;
     dim3 grid(Hkv, B, layer_end - layer_begin);
-    const RowMap rows = {block_table, table_stride, page_rows, num_blocks};
+    const RowMap rows = {block_table, table_stride, page_rows, num_blocks, token_major};
     accept_commit_kernel<<<grid, 256, 0, st>>>(cache_ptrs, layer_begin, draft, target, parents, kv_len, path,
                                                accept_len, bonus, kv_len_out, N, Hkv, D, S_max, status, rows);
     return cudaGetLastError();
@@ -381,9 +384,9 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
 cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,
                              const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
                              int Hkv, int D, int S_max, int* status, cudaStream_t st, const int32_t* block_table,
-                             int table_stride, int page_rows, int num_blocks) {
+                             int table_stride, int page_rows, int num_blocks, int token_major) {
     if (B == 0) return cudaSuccess;
-    const RowMap rmap = {block_table, table_stride, page_rows, num_blocks};
+    const RowMap rmap = {block_table, table_stride, page_rows, num_blocks, token_major};
     cudaLaunchConfig_t cfg = {};
     const int rows_per_block = 128 / (D / 16);
     cfg.gridDim = dim3(N, B, (Hq + 2 * Hkv + rows_per_block - 1) / rows_per_block);

@@ -93,6 +93,7 @@ int vispec_ctx_create(vispec_ctx** out, const vispec_shape* s, int device) {
     c->k_map.resize(s->layers);
     c->page_rows.assign(s->layers, 0);
     c->num_blocks.assign(s->layers, 0);
+    c->token_major.assign(s->layers, 0);
     c->v_map.resize(s->layers);
     *out = c;
     return VISPEC_OK;
@@ -165,10 +166,12 @@ int vispec_cache_register(vispec_ctx* c, int layer, void* k_cache, void* v_cache
     c->h_v[layer] = v_cache;
     c->page_rows[layer] = 0;
     c->num_blocks[layer] = 0;
+    c->token_major[layer] = 0;
     return VISPEC_OK;
 }
 
-int vispec_cache_register_paged(vispec_ctx* c, int layer, void* k_pool, void* v_pool, int num_blocks, int page_rows) {
+int vispec_cache_register_paged(vispec_ctx* c, int layer, void* k_pool, void* v_pool, int num_blocks, int page_rows,
+                                int token_major) {
     if (!c || !k_pool || !v_pool) return VISPEC_E_NULL;
     if (layer < 0 || layer >= c->shape.layers) return VISPEC_E_RANGE;
     if (!aligned(k_pool, 128) || !aligned(v_pool, 128)) return VISPEC_E_ALIGN;
@@ -176,13 +179,22 @@ int vispec_cache_register_paged(vispec_ctx* c, int layer, void* k_pool, void* v_
     if (s.D != 128) return VISPEC_E_UNSUPPORTED;
     if (num_blocks < 1 || (page_rows != 16 && page_rows != 32 && page_rows != 64 && page_rows != 128)) return VISPEC_E_SHAPE;
     if ((long long)num_blocks * s.Hkv >= (1ll << 31)) return VISPEC_E_SHAPE;
-    // 3-D view (d, slot in block, block*head) of a [num_blocks,Hkv,page_rows,D] bf16 pool; one box = 64 d-columns x one
-    // block's slots of one head.  A block number outside the pool reads as zero.
+    if ((long long)num_blocks * page_rows >= (1ll << 31)) return VISPEC_E_SHAPE;
+    // 3-D view of the bf16 pool, one box = 64 d-columns x one block's slots of one head: (d, slot in block, block*head)
+    // for [num_blocks,Hkv,page_rows,D]; (d, head, block*page_rows + slot) for the token-major
+    // [num_blocks,page_rows,Hkv,D].  A block number outside the pool reads as zero.
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return VISPEC_E_CUDA;
-    const cuuint64_t dims[3] = {(cuuint64_t)s.D, (cuuint64_t)page_rows, (cuuint64_t)num_blocks * s.Hkv};
-    const cuuint64_t strides[2] = {(cuuint64_t)s.D * 2, (cuuint64_t)page_rows * s.D * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)page_rows, 1};
+    const cuuint64_t row = (cuuint64_t)s.D * 2;
+    const cuuint64_t dims_h[3] = {(cuuint64_t)s.D, (cuuint64_t)page_rows, (cuuint64_t)num_blocks * s.Hkv};
+    const cuuint64_t dims_t[3] = {(cuuint64_t)s.D, (cuuint64_t)s.Hkv, (cuuint64_t)num_blocks * page_rows};
+    const cuuint64_t strides_h[2] = {row, (cuuint64_t)page_rows * row};
+    const cuuint64_t strides_t[2] = {row, (cuuint64_t)s.Hkv * row};
+    const cuuint32_t box_h[3] = {64, (cuuint32_t)page_rows, 1};
+    const cuuint32_t box_t[3] = {64, 1, (cuuint32_t)page_rows};
+    const cuuint64_t* dims = token_major ? dims_t : dims_h;
+    const cuuint64_t* strides = token_major ? strides_t : strides_h;
+    const cuuint32_t* box = token_major ? box_t : box_h;
     const cuuint32_t estr[3] = {1, 1, 1};
     void* ptrs[2] = {k_pool, v_pool};
     CUtensorMap* maps[2] = {&c->k_map[layer], &c->v_map[layer]};
@@ -199,6 +211,7 @@ int vispec_cache_register_paged(vispec_ctx* c, int layer, void* k_pool, void* v_
     c->h_v[layer] = v_pool;
     c->page_rows[layer] = page_rows;
     c->num_blocks[layer] = num_blocks;
+    c->token_major[layer] = token_major ? 1 : 0;
     return VISPEC_OK;
 }
 
@@ -265,7 +278,7 @@ int vispec_tree_verify_attn_paged(vispec_ctx* c, int layer, const void* q, const
     a.tc5_path = c->tc5_path;
     a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
     a.block_table = block_table; a.table_stride = table_stride;
-    a.page_rows = c->page_rows[layer]; a.num_blocks = c->num_blocks[layer];
+    a.page_rows = c->page_rows[layer]; a.num_blocks = c->num_blocks[layer]; a.token_major = c->token_major[layer];
     if (!attn_tc5_supports(a)) return VISPEC_E_UNSUPPORTED;   // B <= 32, scale > 0, workspace large enough for the table's capacity
     int n = 0;
     cudaError_t err = launch_attn_tc5(a, (cudaStream_t)stream, &n);
@@ -286,12 +299,13 @@ int vispec_kv_compact_paged(vispec_ctx* c, int layer_begin, int layer_end, const
     for (int l = layer_begin; l < layer_end; ++l) {
         if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
         if (!c->page_rows[l]) return VISPEC_E_UNSUPPORTED;
-        if (c->page_rows[l] != pr || c->num_blocks[l] != nb) return VISPEC_E_SHAPE;   // one table serves every layer
+        if (c->page_rows[l] != pr || c->num_blocks[l] != nb || c->token_major[l] != c->token_major[layer_begin])
+            return VISPEC_E_SHAPE;                                                   // one table serves every layer
     }
     if ((long long)table_stride * pr > (1ll << 30)) return VISPEC_E_SHAPE;
     if (launch_kv_compact(c->d_cache_ptrs, layer_begin, layer_end, path, accept_len, kv_len, kv_len_out, B, N, s.Hkv,
                           s.D, table_stride * pr, c->d_status, (cudaStream_t)stream, block_table, table_stride, pr,
-                          nb) != cudaSuccess)
+                          nb, c->token_major[layer_begin]) != cudaSuccess)
         return VISPEC_E_CUDA;
     if (B > 0) c->launches += 1;
     return VISPEC_OK;
@@ -303,7 +317,9 @@ static int paged_range_check(const vispec_ctx* c, int lb, int le, int table_stri
     for (int l = lb; l < le; ++l) {
         if (!c->h_k[l]) return VISPEC_E_UNREGISTERED;
         if (!c->page_rows[l]) return VISPEC_E_UNSUPPORTED;
-        if (c->page_rows[l] != c->page_rows[lb] || c->num_blocks[l] != c->num_blocks[lb]) return VISPEC_E_SHAPE;
+        if (c->page_rows[l] != c->page_rows[lb] || c->num_blocks[l] != c->num_blocks[lb] ||
+            c->token_major[l] != c->token_major[lb])
+            return VISPEC_E_SHAPE;
     }
     if (le > lb && (long long)table_stride * c->page_rows[lb] > (1ll << 30)) return VISPEC_E_SHAPE;
     return VISPEC_OK;
@@ -324,7 +340,8 @@ int vispec_accept_commit_paged(vispec_ctx* c, int layer_begin, int layer_end, co
     const int pr = c->page_rows[layer_begin];
     if (launch_accept_commit(c->d_cache_ptrs, layer_begin, layer_end, draft_ids, target_ids, parents, kv_len, path,
                              accept_len, bonus, kv_len_out, B, N, s.Hkv, s.D, table_stride * pr, c->d_status,
-                             (cudaStream_t)stream, block_table, table_stride, pr, c->num_blocks[layer_begin]) != cudaSuccess)
+                             (cudaStream_t)stream, block_table, table_stride, pr, c->num_blocks[layer_begin],
+                             c->token_major[layer_begin]) != cudaSuccess)
         return VISPEC_E_CUDA;
     if (B > 0) c->launches += 1;
     return VISPEC_OK;
@@ -343,7 +360,7 @@ int vispec_rope_tree_rows_paged(vispec_ctx* c, int layer, void* q, const void* k
     const int pr = c->page_rows[layer];
     if (launch_rope_rows(q, k_new, v_new, positions, kv_len, c->h_k[layer], c->h_v[layer], theta, B, N, s.Hq, s.Hkv,
                          s.D, table_stride * pr, c->d_status, (cudaStream_t)stream, block_table, table_stride, pr,
-                         c->num_blocks[layer]) != cudaSuccess)
+                         c->num_blocks[layer], c->token_major[layer]) != cudaSuccess)
         return VISPEC_E_CUDA;
     if (B > 0) c->launches += 1;
     return VISPEC_OK;

@@ -17,6 +17,7 @@ struct vispec_ctx {
     std::vector<void*> h_k, h_v;    // host copy of the registered pointers
     std::vector<CUtensorMap> k_map, v_map;  // TMA descriptors per layer (D == 128 only)
     std::vector<int> page_rows, num_blocks; // per layer: slots per pool block (0 = contiguous cache), pool blocks
+    std::vector<int> token_major;           // per layer: pool is [block][slot][head][D] instead of [block][head][slot][D]
     void* ws = nullptr;             // caller-owned workspace
     size_t ws_bytes = 0;
     uint64_t launches = 0;
@@ -45,20 +46,20 @@ cudaError_t launch_kv_compact(void* const* cache_ptrs, int layer_begin, int laye
                               const int32_t* path, const int32_t* accept_len, const int32_t* kv_len,
                               int32_t* kv_len_out, int B, int N, int Hkv, int D, int S_max, int* status,
                               cudaStream_t st, const int32_t* block_table = nullptr, int table_stride = 0,
-                              int page_rows = 0, int num_blocks = 0);
+                              int page_rows = 0, int num_blocks = 0, int token_major = 0);
 
 cudaError_t launch_accept_commit(void* const* cache_ptrs, int layer_begin, int layer_end, const int32_t* draft,
                                  const int32_t* target, const int32_t* parents, const int32_t* kv_len,
                                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, int B, int N,
                                  int Hkv, int D, int S_max, int* status, cudaStream_t st,
                                  const int32_t* block_table = nullptr, int table_stride = 0, int page_rows = 0,
-                                 int num_blocks = 0);
+                                 int num_blocks = 0, int token_major = 0);
 
 cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,
                              const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
                              int Hkv, int D, int S_max, int* status, cudaStream_t st,
                              const int32_t* block_table = nullptr, int table_stride = 0, int page_rows = 0,
-                             int num_blocks = 0);
+                             int num_blocks = 0, int token_major = 0);
 
 cudaError_t launch_accept_sampled(const int32_t* draft_ids, const int32_t* parents, const float* p, const float* p_hat,
                                   const float* u_accept, const float* u_bonus, int B, int N, int V, int32_t* path,
@@ -82,7 +83,7 @@ struct AttnArgs {
     const CUtensorMap* k_map; const CUtensorMap* v_map;
     // paged cache (page_rows != 0): pool blocks of page_rows slots, block_table [B][table_stride]; S_max is then
     // table_stride * page_rows
-    const int32_t* block_table; int table_stride, page_rows, num_blocks;
+    const int32_t* block_table; int table_stride, page_rows, num_blocks, token_major;
 };
 // Generic split-KV kernel on warp-level tensor-core instructions (any supported shape).
 cudaError_t init_attn_generic();   // once per device, with that device current

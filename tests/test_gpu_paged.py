@@ -40,7 +40,7 @@ def _unpage(pool, table, S_max):
     return blocks.reshape(B, Hkv, per * rows, D)[:, :, :S_max]
 
 
-def _run_paged(q, pools, table, kv_len, mask, scale, split_form=0, N_max=None):
+def _run_paged(q, pools, table, kv_len, mask, scale, split_form=0, N_max=None, token_major=False):
     from paper_2509_15235_b200 import binding
     import gpu_util as gu
     B, N, Hq, D = q.shape
@@ -48,8 +48,10 @@ def _run_paged(q, pools, table, kv_len, mask, scale, split_form=0, N_max=None):
     ctx = binding.VerifyContext(max(B, 1), N_max or N, Hq, Hkv, D, table.shape[1] * rows, 1)
     if split_form:
         ctx.ctx_set_option(binding.OPT_SPLIT_FORM, split_form)
+    if token_major:
+        pools = [np.ascontiguousarray(x.transpose(0, 2, 1, 3)) for x in pools]
     kd, vd = gu.bf16_dev(pools[0]), gu.bf16_dev(pools[1])
-    ctx.cache_register_paged(0, kd, vd)
+    ctx.cache_register_paged(0, kd, vd, token_major)
     out = torch.full((B, N, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
     lse = torch.full((B, Hq, N), float("nan"), dtype=torch.float32, device="cuda")
     ctx.tree_verify_attn_paged(0, gu.bf16_dev(q), gu.i32_dev(kv_len), gu.i32_dev(table), gu.u64_dev(mask), scale, out, lse)
@@ -73,7 +75,8 @@ def _case(B, N, Hq, Hkv, S_list, S_max, seed):
 
 @pytest.mark.parametrize("page_rows", [16, 32, 64, 128])
 @pytest.mark.parametrize("split_form", [0, 1, 2, 3])
-def test_paged_attention_equals_contiguous_and_oracle(page_rows, split_form):
+@pytest.mark.parametrize("token_major", [False, True])
+def test_paged_attention_equals_contiguous_and_oracle(page_rows, split_form, token_major):
     import gpu_util as gu
     B, N, Hq, Hkv, S_max = 3, 60, 8, 2, 1152
     q, k, v, kv_len, mask, rng = _case(B, N, Hq, Hkv, [1000, 707, 3], S_max, 100 + page_rows)
@@ -84,7 +87,7 @@ def test_paged_attention_equals_contiguous_and_oracle(page_rows, split_form):
     for b in range(B):
         first_unused = -(-(int(kv_len[b]) + N) // page_rows)
         table[b, first_unused:] = 2 ** 30
-    out, lse, status = _run_paged(q, pools, table, kv_len, mask, scale, split_form)
+    out, lse, status = _run_paged(q, pools, table, kv_len, mask, scale, split_form, token_major=token_major)
     assert status == 0 and not np.isnan(out).any()
     want, want_lse = oracle.tree_attn(q, k, v, kv_len, mask, scale)
     assert np.abs(out - want).max() <= TOL and np.abs(lse - want_lse).max() <= LSE_TOL
@@ -173,7 +176,8 @@ def test_paged_commit_matches_the_oracle_on_the_logical_cache():
     ctx.close()
 
 
-def test_paged_accept_commit_and_rope_match_the_oracle():
+@pytest.mark.parametrize("token_major", [False, True])
+def test_paged_accept_commit_and_rope_match_the_oracle(token_major):
     from paper_2509_15235_b200 import binding
     import gpu_util as gu
     cfg = synth.get_config("paper_tree")
@@ -190,10 +194,13 @@ def test_paged_accept_commit_and_rope_match_the_oracle():
     for l in range(layers):
         k = synth.normal_bf16((B, Hkv, S_max, D), 300 + l); v = synth.normal_bf16((B, Hkv, S_max, D), 310 + l)
         pools, table = _page((k, v), rows, np.random.Generator(np.random.Philox(32)))
+        if token_major:
+            pools = [np.ascontiguousarray(x.transpose(0, 2, 1, 3)) for x in pools]
         kd, vd = gu.bf16_dev(pools[0]), gu.bf16_dev(pools[1])
-        ctx.cache_register_paged(l, kd, vd)
+        ctx.cache_register_paged(l, kd, vd, token_major)
         state.append([k, v, kd, vd])
     tab_d = gu.i32_dev(table)
+    pool_bits = (lambda t: gu.bf16_bits(t).transpose(0, 2, 1, 3)) if token_major else gu.bf16_bits   # back to [block, head, slot, D]
     # RoPE + placement on every layer, then acceptance + commit over both layers in one launch
     for l in range(layers):
         q = synth.normal_bf16((B, N, Hq, D), 320 + l); kn = synth.normal_bf16((B, N, Hkv, D), 330 + l)
@@ -203,7 +210,7 @@ def test_paged_accept_commit_and_rope_match_the_oracle():
         wq, wk, wv, skipped = oracle.rope_rows(q, kn, vn, positions, kv_len, state[l][0], state[l][1], 1e4)
         assert skipped == 0
         torch.cuda.synchronize()
-        gk = _unpage(gu.bf16_bits(state[l][2]), table, S_max); gv = _unpage(gu.bf16_bits(state[l][3]), table, S_max)
+        gk = _unpage(pool_bits(state[l][2]), table, S_max); gv = _unpage(pool_bits(state[l][3]), table, S_max)
         assert np.array_equal(gv, wv)
         step = np.abs(gk.astype(np.int32) - wk.astype(np.int32))          # bit patterns of equal sign: steps
         assert step.max() <= 1 and (step != 0).mean() <= 1e-4
@@ -221,8 +228,8 @@ def test_paged_accept_commit_and_rope_match_the_oracle():
     assert np.array_equal(bonus.cpu().numpy(), wb) and (wl > 1).any()
     for l in range(layers):
         wk, wv, wn = oracle.kv_compact(state[l][0], state[l][1], wp, wl, kv_len)
-        assert np.array_equal(_unpage(gu.bf16_bits(state[l][2]), table, S_max), wk)
-        assert np.array_equal(_unpage(gu.bf16_bits(state[l][3]), table, S_max), wv)
+        assert np.array_equal(_unpage(pool_bits(state[l][2]), table, S_max), wk)
+        assert np.array_equal(_unpage(pool_bits(state[l][3]), table, S_max), wv)
         assert np.array_equal(new_len.cpu().numpy(), wn)
     ctx.close()
 
