@@ -111,7 +111,7 @@ typedef enum vispec_option {
      * whenever the shape allows one cluster per (sequence, kv head, row block); 3 is 1 with the second kernel
      * always.  The in-kernel merge counts arrivals in the first 64 KiB of the workspace, which
      * vispec_ctx_set_workspace zeroes and every call leaves zero (a call that ended with VISPEC_E_TIMEOUT may
-     * not: set the workspace again after one). */
+     * not: vispec_status_poll zeroes them again when it reports that code). */
     VISPEC_OPT_SPLIT_FORM = 3
 } vispec_option;
 
@@ -326,7 +326,8 @@ int vispec_accept_commit(vispec_ctx* ctx, int layer_begin, int layer_end, const 
                          int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, void* stream);
 
 /* Read and clear the device status word (synchronises `stream`; not a hot call).
- * `*code` (host) receives VISPEC_OK or the first asynchronous error recorded since the last poll. */
+ * `*code` (host) receives VISPEC_OK or the first asynchronous error recorded since the last poll.  When that
+ * is VISPEC_E_TIMEOUT the arrival counters at the head of the workspace are zeroed on `stream` as well. */
 int vispec_status_poll(vispec_ctx* ctx, int* code /*host*/, void* stream);
 
 /* Number of kernels the library has launched through this context since creation (host counter). */

@@ -490,6 +490,8 @@ int vispec_status_poll(vispec_ctx* c, int* code, void* stream) {
     if (cudaMemcpyAsync(&v, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return VISPEC_E_CUDA;
     if (cudaMemsetAsync(c->d_status, 0, sizeof(int), st) != cudaSuccess) return VISPEC_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return VISPEC_E_CUDA;
+    // a call that gave up on a wait may have left arrival counters behind: the next call finds them zero again
+    if (v == VISPEC_E_TIMEOUT && c->ws && cudaMemsetAsync(c->ws, 0, kCounterBytes, st) != cudaSuccess) return VISPEC_E_CUDA;
     *code = v;
     return VISPEC_OK;
 }
