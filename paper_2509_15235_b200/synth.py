@@ -231,10 +231,11 @@ def make_sampled_inputs(parents: np.ndarray, V: int, seed: int, sharpness: float
 
 def make_rerank_candidates(B: int, depth: int, width: int, vocab: int, seed: int) -> Dict[str, np.ndarray]:
     """Candidates of a level-by-level tree expansion (the input of the rerank): level 1 holds `width` children
-    of the root, every later level `width` children of each of the `width` best candidates of the level before
-    (best by cumulative score), so M = width + (depth - 1) * width^2 (136 for depth 3, width 8).  A child's score
-    is its parent's plus the log of one of the `width` largest entries of a random distribution over the
-    vocabulary (softmax of 3 * N(0,1)); its token is that entry's index."""
+    of the root, every later level `width` children of each of `width` candidates of the level before (drawn at
+    random: which ones a draft model would expand is its business, not this generator's), so
+    M = width + (depth - 1) * width^2 (136 for depth 3, width 8).  A child's score is its parent's plus the log
+    of its share of a random split of the unit mass into width + 1 parts (cubed exponentials: a few children carry
+    most of it, the last part stands for the rest of the vocabulary); tokens are distinct random ids."""
     rng = _rng(seed)
     M = width + (depth - 1) * width * width
     parent = np.full((B, M), -1, dtype=np.int32)
@@ -242,9 +243,10 @@ def make_rerank_candidates(B: int, depth: int, width: int, vocab: int, seed: int
     score = np.zeros((B, M), dtype=np.float32)
 
     def expand():
-        pr = softmax_rows_f32(np.float32(3.0) * rng.standard_normal((1, vocab), dtype=np.float32))[0]
-        top = np.argsort(-pr, kind="stable")[:width]
-        return top.astype(np.int32), np.log(pr[top]).astype(np.float32)
+        w = rng.standard_exponential(width + 1) ** 3
+        share = (w / w.sum())[:width]
+        tok = rng.choice(vocab, size=width, replace=False)
+        return tok.astype(np.int32), np.log(np.maximum(share, 1e-30)).astype(np.float32)
 
     for b in range(B):
         tok, lp = expand()
@@ -252,7 +254,7 @@ def make_rerank_candidates(B: int, depth: int, width: int, vocab: int, seed: int
         level = list(range(width))
         n = width
         for _ in range(1, depth):
-            best = sorted(level, key=lambda i: (-float(score[b, i]), i))[:width]
+            best = [level[j] for j in rng.permutation(len(level))[:width]]
             level = []
             for par in sorted(best):
                 tok, lp = expand()
