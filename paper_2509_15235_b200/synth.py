@@ -218,13 +218,13 @@ def make_sampled_inputs(parents: np.ndarray, V: int, seed: int, sharpness: float
         ph[b] = softmax_rows_f32(np.float32(sharpness) * g)
     ids = np.zeros((B, N), dtype=np.int32)
     for b in range(B):
-        cdfs: Dict[int, np.ndarray] = {}
+        rows: Dict[int, np.ndarray] = {}
         for i in range(1, N):
             par = int(parents[b, i])
-            if par not in cdfs:
-                cdfs[par] = np.cumsum(ph[b, par].astype(np.float64))
-            cdf = cdfs[par]
-            ids[b, i] = min(int(np.searchsorted(cdf, rng.random() * cdf[-1], side="right")), V - 1)
+            if par not in rows:
+                w = ph[b, par].astype(np.float64)
+                rows[par] = w / w.sum()
+            ids[b, i] = int(rng.choice(V, p=rows[par]))
     return {"p_target": p, "p_draft": ph, "draft_ids": ids,
             "u_accept": rng.random((B, N), dtype=np.float32), "u_bonus": rng.random(B, dtype=np.float32)}
 
