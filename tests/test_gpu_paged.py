@@ -95,6 +95,24 @@ def test_paged_attention_equals_contiguous_and_oracle(page_rows, split_form, tok
     assert st == 0 and np.array_equal(out, ref) and np.array_equal(lse, ref_lse)
 
 
+@pytest.mark.parametrize("B,N,Hq,Hkv,S_list,S_max,page_rows,token_major", [
+    (2, 128, 8, 1, [200, 77], 384, 32, False),       # largest tree: 1024 query rows per kv head, two mask words
+    (2, 1, 4, 2, [129, 0], 256, 16, True),           # a single node (plain decode step); an empty prefix
+    (32, 9, 2, 2, list(range(3, 35)), 128, 64, False),   # the most sequences a call takes
+    (3, 65, 3, 3, [130, 64, 1], 256, 128, True),     # two mask words with one head per kv head
+])
+def test_paged_attention_edge_shapes(B, N, Hq, Hkv, S_list, S_max, page_rows, token_major):
+    q, k, v, kv_len, mask, rng = _case(B, N, Hq, Hkv, S_list, S_max, 500 + B + N)
+    pools, table = _page((k, v), page_rows, rng)
+    scale = 1 / math.sqrt(128)
+    out, lse, status = _run_paged(q, pools, table, kv_len, mask, scale, token_major=token_major)
+    want, want_lse = oracle.tree_attn(q, k, v, kv_len, mask, scale)
+    assert status == 0 and not np.isnan(out).any()
+    assert np.abs(out - want).max() <= TOL
+    finite = np.isfinite(want_lse)
+    assert np.array_equal(np.isfinite(lse), finite) and np.abs(lse[finite] - want_lse[finite]).max() <= LSE_TOL
+
+
 def test_paged_attention_rows_past_the_end_may_hold_anything():
     B, N, Hq, Hkv, S_max = 2, 31, 4, 4, 512
     q, k, v, kv_len, mask, rng = _case(B, N, Hq, Hkv, [300, 129], S_max, 7)
