@@ -285,9 +285,14 @@ class DeviceWorkload:
 class HostStep:
     """End-to-end step: the cycle's inputs start in pinned host memory and its results end there.
     Per step: H2D of parents / draft_ids / target_ids / kv_len, of q for all layers and of the tree's
-    new K/V rows for all layers (written to slots S..S+N-1 of the resident caches); D2H of the
-    attention output of all layers, the accepted path, accept_len, bonus and the new kv_len.
-    The committed prefix of the cache is state that lives on the device across cycles."""
+    new K/V rows for all layers; D2H of the attention output of all layers, the accepted path, accept_len,
+    bonus and the new kv_len.  The committed prefix of the cache is state that lives on the device across cycles.
+    The layers go in four groups: while one group's attention runs, the next group's inputs arrive on a second
+    stream and the previous group's outputs leave on a third (PCIe carries both directions at once).  The tree's
+    rows are put behind the committed prefix by vispec_rope_tree_rows with all positions 0 (the identity rotation:
+    the synthetic rows stand for rows that are already rotated)."""
+
+    GROUPS = 4
 
     def __init__(self, wl: DeviceWorkload, tree, per_layer):
         torch = wl.torch
@@ -298,11 +303,11 @@ class HostStep:
         self.h_out = pin(torch.zeros_like(self.h_q))
         S = tree["kv_len"]
         N = cfg.N
-        # new rows [L,B,Hkv,N,D] gathered from the synthetic caches (host side, outside the timed region)
-        rows_k = np.stack([np.stack([x["k_cache"][b, :, S[b]:S[b] + N] for b in range(cfg.B)]) for x in per_layer])
-        rows_v = np.stack([np.stack([x["v_cache"][b, :, S[b]:S[b] + N] for b in range(cfg.B)]) for x in per_layer])
-        self.h_newk = pin(torch.from_numpy(rows_k.view(np.int16)).view(torch.bfloat16))
-        self.h_newv = pin(torch.from_numpy(rows_v.view(np.int16)).view(torch.bfloat16))
+        # new rows [L,B,N,Hkv,D] gathered from the synthetic caches (host side, outside the timed region)
+        rows_k = np.stack([np.stack([x["k_cache"][b, :, S[b]:S[b] + N].transpose(1, 0, 2) for b in range(cfg.B)]) for x in per_layer])
+        rows_v = np.stack([np.stack([x["v_cache"][b, :, S[b]:S[b] + N].transpose(1, 0, 2) for b in range(cfg.B)]) for x in per_layer])
+        self.h_newk = pin(torch.from_numpy(np.ascontiguousarray(rows_k).view(np.int16)).view(torch.bfloat16))
+        self.h_newv = pin(torch.from_numpy(np.ascontiguousarray(rows_v).view(np.int16)).view(torch.bfloat16))
         self.d_newk = torch.empty_like(self.h_newk, device=wl.dev)
         self.d_newv = torch.empty_like(self.h_newv, device=wl.dev)
         self.h_ints = pin(torch.from_numpy(np.concatenate([tree["parents"].ravel(), tree["draft_ids"].ravel(),
@@ -313,34 +318,47 @@ class HostStep:
                       self.d_ints[2 * BN:3 * BN].view(cfg.B, N), self.d_ints[3 * BN:])
         self.d_res = torch.zeros(BN + 3 * cfg.B, dtype=torch.int32, device=wl.dev)
         self.h_res = pin(torch.zeros(BN + 3 * cfg.B, dtype=torch.int32))
-        self.S = [int(s) for s in S]
+        self.pos0 = torch.zeros((cfg.B, N), dtype=torch.int32, device=wl.dev)
         self.h2d = (self.h_q.numel() + self.h_newk.numel() + self.h_newv.numel()) * 2 + self.h_ints.numel() * 4
         self.d2h = self.h_out.numel() * 2 + self.h_res.numel() * 4
+        g = max(1, min(self.GROUPS, wl.L))
+        edges = [round(i * wl.L / g) for i in range(g + 1)]
+        self.groups = [(edges[i], edges[i + 1]) for i in range(g) if edges[i + 1] > edges[i]]
+        self.s_in, self.s_out = torch.cuda.Stream(device=wl.dev), torch.cuda.Stream(device=wl.dev)
+        self.ev_in = [torch.cuda.Event() for _ in self.groups]
+        self.ev_done = [torch.cuda.Event() for _ in self.groups]
 
     def step(self):
         wl, cfg = self.wl, self.wl.cfg
         torch = wl.torch
         B, N = cfg.B, cfg.N
+        main = torch.cuda.current_stream()
+        self.s_in.wait_stream(main)                 # the previous step has let go of the input buffers
+        with torch.cuda.stream(self.s_in):
+            for i, (lo, hi) in enumerate(self.groups):
+                wl.q[lo:hi].copy_(self.h_q[lo:hi], non_blocking=True)
+                self.d_newk[lo:hi].copy_(self.h_newk[lo:hi], non_blocking=True)
+                self.d_newv[lo:hi].copy_(self.h_newv[lo:hi], non_blocking=True)
+                self.ev_in[i].record(self.s_in)
         self.d_ints.copy_(self.h_ints, non_blocking=True)
-        wl.q.copy_(self.h_q, non_blocking=True)
-        self.d_newk.copy_(self.h_newk, non_blocking=True)
-        self.d_newv.copy_(self.h_newv, non_blocking=True)
         parents, draft, target, kv_len = self.views
-        for l in range(wl.L):                      # place the tree's rows behind the committed prefix
-            for b in range(B):
-                s = self.S[b]
-                wl.k[l][b, :, s:s + N].copy_(self.d_newk[l, b], non_blocking=True)
-                wl.v[l][b, :, s:s + N].copy_(self.d_newv[l, b], non_blocking=True)
         c = wl.ctx
         path = self.d_res[:B * N].view(B, N)
         alen, bonus, new_len = self.d_res[B * N:B * N + B], self.d_res[B * N + B:B * N + 2 * B], self.d_res[B * N + 2 * B:]
         c.tree_mask_build(parents, wl.mask, wl.depth)
-        for l in range(wl.L):
-            c.tree_verify_attn(l, wl.q[l], kv_len, wl.mask, wl.scale, wl.out[l])
+        for i, (lo, hi) in enumerate(self.groups):
+            main.wait_event(self.ev_in[i])
+            for l in range(lo, hi):
+                c.rope_tree_rows(l, wl.q[l], self.d_newk[l], self.d_newv[l], self.pos0, kv_len, 1e4)   # placement
+                c.tree_verify_attn(l, wl.q[l], kv_len, wl.mask, wl.scale, wl.out[l])
+            self.ev_done[i].record(main)
+            self.s_out.wait_event(self.ev_done[i])
+            with torch.cuda.stream(self.s_out):
+                self.h_out[lo:hi].copy_(wl.out[lo:hi], non_blocking=True)
         c.accept_commit(0, wl.L, draft, target, parents, kv_len, path, alen, bonus, new_len)
-        self.h_out.copy_(wl.out, non_blocking=True)
         self.h_res.copy_(self.d_res, non_blocking=True)
-        torch.cuda.current_stream().synchronize()      # the caller reads accept_len to go on
+        main.synchronize()                           # the caller reads accept_len to go on
+        self.s_out.synchronize()
 
 
 # ------------------------------------------------------------------------------------ oracle legs
@@ -354,12 +372,14 @@ def oracle_sample(cfg, tree, layers, budget_heads):
     t0 = time.perf_counter()
     mask, _, _ = oracle.tree_mask(tree["parents"])
     path, alen, _ = oracle.accept(tree["draft_ids"], tree["target_ids"], tree["parents"])
+    outs = []
     for x in layers:
         q, k, v = x["q"][:, :, :hk * G], x["k_cache"][:, :hk], x["v_cache"][:, :hk]
-        oracle.tree_attn(q, k, v, tree["kv_len"], mask, 1.0 / math.sqrt(cfg.D), want_lse=False)
+        outs.append(oracle.tree_attn(q, k, v, tree["kv_len"], mask, 1.0 / math.sqrt(cfg.D), want_lse=False)[0])
         oracle.kv_compact(k, v, path, alen, tree["kv_len"])
     dt = time.perf_counter() - t0
     kv_bytes = len(layers) * int(sum(2 * (int(s) + cfg.N) * hk * cfg.D * 2 for s in tree["kv_len"]))
+    oracle_sample.last = {"outs": outs, "accept_len": alen, "heads": hk * G}
     return kv_bytes / dt / 1e9, dt, hk, oracle.num_threads()
 
 
@@ -596,6 +616,15 @@ def main():
     if not args.no_cpu_baseline:
         n_l = L
         gbs, dt, hk, cores = oracle_sample(cfg, tree, per_layer[:n_l], cfg.Hkv)
+        if e2e:
+            # the last end-to-end step's host-side results against what the oracle has just computed from the same inputs
+            ref = oracle_sample.last
+            got = hs.h_out.float().numpy()
+            err = max(float(np.abs(got[l][:, :, :ref["heads"]] - o).max()) for l, o in enumerate(ref["outs"]))
+            got_len = hs.h_res[cfg.B * cfg.N:cfg.B * cfg.N + cfg.B].numpy()
+            if err > 2e-2 or not np.array_equal(got_len, ref["accept_len"]):
+                raise RuntimeError(f"end-to-end results differ from the oracle: max abs err {err}, accept_len {got_len}")
+            e2e["checked_against_oracle"] = {"layers": len(ref["outs"]), "max_abs_err": err}
         line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
                                 "sample": f"one step: {n_l} of {L} layers, {hk} of {cfg.Hkv} kv heads, all nodes, full KV "
                                           f"length, plus mask/accept/commit ({dt:.1f} s of fp64 C + OpenMP)"}
