@@ -1108,6 +1108,12 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         __syncwarp();
         cluster_sync_all();
         TRACE_MISC(13);
+        if (warp == 1) {
+            // every thread of the CTA is past its last tensor-memory access: give the columns back now, beside the
+            // merge, instead of on the way out
+            tc_fence_after();
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
+        }
         if (warp >= 4 && !*abort_flag) {
         const int rp = (ROWS + ck - 1) / ck;
         const int row0 = cr * rp;
@@ -1174,7 +1180,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     // CTA gets here (all its other waits are bounded), so this hardware barrier ends.
     if (CL) cluster_sync_all();
     TRACE_MISC(9);
-    if (warp == 1) {
+    if (!CL && warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
     }
