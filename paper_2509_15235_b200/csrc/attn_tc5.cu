@@ -306,14 +306,15 @@ struct Tc5Params {
 
 // ---- schedule ---------------------------------------------------------------------------------------
 // Built by one full warp.  Reads kv_len only.
-__device__ void sched_build(Sched& s, const Tc5Params& p, int lane) {
+__device__ void sched_build(Sched& s, const Tc5Params& p, int lane, int kv_first) {   // kv_first: kv_len[lane], fetched by the caller
+
     const int upb = p.Hkv * p.n_mblocks;        // units per sequence
     int carry = 0;
     for (int b0 = 0; b0 < p.B; b0 += 32) {
         const int b = b0 + lane;
         int st = 0, S = 0;
         if (b < p.B) {
-            S = p.kv_len[b];
+            S = b0 == 0 ? kv_first : p.kv_len[b];
             const bool ok = (S >= 0 && S + p.N <= p.S_max);
             st = ok ? (S + p.N + STEP - 1) / STEP : 0;
             s.steps[b] = st;
@@ -558,6 +559,10 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
     extern __shared__ __align__(1024) unsigned char sm[];
     TRACE_MISC(0);
+    // the schedule hangs on kv_len, and a CTA that starts after its predecessor kernel has ended hangs on the
+    // schedule: the load goes out first
+    int kv_first = 0;
+    if (p.early && threadIdx.x >= 96 && threadIdx.x < 128 && (int)threadIdx.x - 96 < p.B) kv_first = p.kv_len[threadIdx.x - 96];
     if (threadIdx.x == 0) TL_START(p.trace_idx, 0);
     CTA_T(0);
     const uint32_t base = smem_u32(sm);
@@ -596,9 +601,12 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (warp == 3) sched_build(sched, p, lane);
     pdl_launch_dependents();
-    if (!p.early) pdl_wait();
+    if (!p.early) {                                          // nothing is read before the preceding kernel has ended
+        pdl_wait();
+        if (warp == 3 && lane < p.B) kv_first = p.kv_len[lane];
+    }
+    if (warp == 3) sched_build(sched, p, lane, kv_first);
     TRACE_MISC(1);
     tc_fence_before();
     __syncthreads();
@@ -1302,7 +1310,7 @@ stream_probe_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_cons
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) sched_build(sched, p, lane);
+    if (warp == 1) sched_build(sched, p, lane, lane < p.B ? p.kv_len[lane] : 0);
     pdl_launch_dependents();
     if (!p.early) pdl_wait();
     __syncthreads();
