@@ -39,9 +39,9 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one attention launch of the benchmarked workload, from the ncu
 # capture summarised under profiles/; None until a capture exists.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    "llava7b": 66_235_000,                # profiles/attn_tc5_kernel_llava7b.md: 65.58 MB read + 0.66 MB written
-    "llava13b_b4": 335_310_000,           # profiles/attn_tc5_kernel_llava13b_b4.md (attention kernel; its merge kernel adds 9.5 MB)
-    "qwen3b_S32768_N16_B8": 274_600_000,  # profiles/attn_tc5_kernel_qwen3b_S32768_N16_B8.md (merge kernel adds 9.6 MB)
+    "llava7b": 66_345_000,                # profiles/attn_tc5_kernel_llava7b.md: 65.58 MB read + 0.77 MB written
+    "llava13b_b4": 335_470_000,           # profiles/attn_tc5_kernel_llava13b_b4.md: 330.22 MB read + 5.25 MB written
+    "qwen3b_S32768_N16_B8": 274_550_000,  # profiles/attn_tc5_kernel_qwen3b_S32768_N16_B8.md (merge kernel adds 9.6 MB)
 }
 
 
