@@ -13,6 +13,14 @@
  *   vispec_accept            greedy (temperature 0) acceptance walk -> accepted path, bonus token
  *   vispec_kv_compact        gather the accepted path's K/V rows into the contiguous cache
  *
+ * and the steps next to it in a decoding cycle:
+ *
+ *   vispec_accept_commit     acceptance and commit in one launch
+ *   vispec_tree_rerank       keep the K best-scored candidates of the tree expansion (App. A) as the tree
+ *   vispec_rope_tree_rows    rotary embedding of the tree's q/k rows and their placement in the cache
+ *   vispec_accept_sampled    acceptance at temperature > 0 (Sec. 3.1's min(1, p/p^) rule with residual resampling)
+ *   vispec_cache_register_paged and the *_paged calls: the same work on a pool of cache blocks and a block table
+ *
  * Conventions
  *   - Every pointer is a DEVICE pointer unless its comment says "host".  The library never takes
  *     ownership of caller memory and never frees it.
