@@ -279,3 +279,24 @@ def test_stream_probe_runs_and_validates_its_arguments(gu):
     with pytest.raises(binding.VispecError) as e:
         ctx64.stream_probe(0, gu.i32_dev([10]), 8)
     assert e.value.code == -5                                   # D = 64: no TMA maps
+
+
+def test_seeded_random_shapes_against_the_oracle(gu):
+    """Sixty seeded draws of (batch, heads, group size, tree size, lengths, split form): every output element
+    against the oracle.  Lengths straddle tile boundaries; some sequences are empty."""
+    rng = np.random.Generator(np.random.Philox(2024))
+    for case in range(60):
+        B = int(rng.integers(1, 6))
+        Hkv = int(rng.choice([1, 2, 3, 4, 8]))
+        G = int(rng.choice([1, 2, 4, 7, 8]))
+        N = int(rng.choice([1, 2, 7, 16, 31, 60, 64, 65, 100, 128]))
+        S_hi = int(rng.choice([0, 5, 127, 128, 129, 400, 1000, 1400]))
+        kv_len = rng.integers(0, S_hi + 1, size=B).astype(np.int32)
+        S_max = (int(kv_len.max()) + N + 127) // 128 * 128 + int(rng.choice([0, 128]))
+        split_form = int(rng.integers(0, 4))
+        q = synth.normal_bf16((B, N, Hkv * G, 128), 9000 + 3 * case)
+        k = synth.normal_bf16((B, Hkv, S_max, 128), 9001 + 3 * case)
+        v = synth.normal_bf16((B, Hkv, S_max, 128), 9002 + 3 * case)
+        parents = np.stack([synth.draw_tree(N, 8, 0, rng) for _ in range(B)])
+        mask, _, _ = oracle.tree_mask(parents)
+        _check(gu, q, k, v, kv_len, mask, 1 / math.sqrt(128), split_form=split_form)
