@@ -55,7 +55,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
-    ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context: 0 automatic, 1 partials + merge kernel, 2 clusters")
+    ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context (0 automatic; see vispec.h)")
     ap.add_argument("--no-sampled", action="store_true", help="skip the timing of vispec_accept_sampled")
     ap.add_argument("--paged", type=int, default=0, help="serve the caches from a block pool of this many slots per block (16/32/64/128)")
     ap.add_argument("--token-major", action="store_true", help="with --paged: pool blocks are [slots, kv heads, D] instead of [kv heads, slots, D]")

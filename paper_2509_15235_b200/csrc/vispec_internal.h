@@ -23,7 +23,7 @@ struct vispec_ctx {
     uint64_t launches = 0;
     bool force_generic = false;     // VISPEC_OPT_FORCE_GENERIC (or VISPEC_FORCE_GENERIC=1 at context creation)
     bool early_prefetch = true;     // VISPEC_OPT_EARLY_PREFETCH
-    int tc5_path = 0;               // VISPEC_OPT_SPLIT_FORM: 0 automatic, 1 partials in global memory, 2 clusters
+    int tc5_path = 0;               // VISPEC_OPT_SPLIT_FORM: 0 automatic, 1 partials in global memory, 2 clusters, 3 merge kernel always
 };
 
 namespace vispec {
@@ -79,7 +79,7 @@ struct AttnArgs {
     int* status;
     int sm_count;
     bool early_prefetch;   // committed-prefix tiles may be read before the preceding kernel has completed
-    int tc5_path;          // 0 automatic, 1 partials in global memory + merge kernel, 2 clusters where possible
+    int tc5_path;          // 0 automatic, 1 partials in global memory (3: merge kernel always), 2 clusters where possible
     const CUtensorMap* k_map; const CUtensorMap* v_map;
     // paged cache (page_rows != 0): pool blocks of page_rows slots, block_table [B][table_stride]; S_max is then
     // table_stride * page_rows
