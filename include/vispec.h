@@ -59,7 +59,8 @@ typedef enum vispec_status {
     VISPEC_E_TIMEOUT = -7,      /* a bounded device-side wait gave up (status word only) */
     VISPEC_E_BAD_TREE = -8,     /* parents[b][i] not in [0,i) for i>0, or parents[b][0] != -1 */
     VISPEC_E_UNREGISTERED = -9, /* layer has no registered cache, or pointers differ from it */
-    VISPEC_E_WORKSPACE = -10    /* workspace missing or too small */
+    VISPEC_E_WORKSPACE = -10,   /* workspace missing or too small */
+    VISPEC_E_POSITIONS = -11    /* positions differ from kv_len + depth (status word, VISPEC_OPT_CHECK_POSITIONS) */
 } vispec_status;
 
 #define VISPEC_MAX_TREE_NODES 128
@@ -105,9 +106,14 @@ typedef enum vispec_option {
      * `stream` is still running (programmatic dependent launch).  Before that kernel has completed it
      * reads only kv_len and cache tiles that lie wholly inside the committed prefix [0, S) - state that
      * the previous decoding cycle committed; q, tree_mask, the tree's own K/V rows (slots S..S+N-1) are
-     * read, and everything is written, only after it has completed.  Set 0 if the kernel enqueued
-     * immediately before an attention call writes kv_len or committed cache slots (for instance
-     * vispec_kv_compact directly followed by attention): then nothing is read early. */
+     * read, and everything is written, only after it has completed.  Attention calls (and the stream probe) let
+     * their successor start as soon as they have started themselves, so through a run of back-to-back attention
+     * calls the early reads of a later call may overlap the kernel that preceded the first of them.  The rule:
+     * a kernel that writes kv_len or committed cache slots (vispec_kv_compact, vispec_accept_commit) must be
+     * followed by at least one kernel that does not start early - vispec_tree_mask_build, vispec_rope_tree_rows
+     * (it waits for its predecessor before it lets its successor in) or any ordinary kernel - before the next
+     * attention call with this option on; the decoding cycle (commit, mask build, attention x layers) satisfies
+     * it.  Otherwise set 0 for the attention calls in between: then nothing is read early. */
     VISPEC_OPT_EARLY_PREFETCH = 1,
     /* Default 0 (1 if the environment has VISPEC_FORCE_GENERIC=1 at context creation).  Route attention
      * through the shape-generic warp-level kernel even where the TMA/tcgen05 kernel applies. */
@@ -120,7 +126,18 @@ typedef enum vispec_option {
      * always.  The in-kernel merge counts arrivals in the first 64 KiB of the workspace, which
      * vispec_ctx_set_workspace zeroes and every call leaves zero (a call that ended with VISPEC_E_TIMEOUT may
      * not: vispec_status_poll zeroes them again when it reports that code). */
-    VISPEC_OPT_SPLIT_FORM = 3
+    VISPEC_OPT_SPLIT_FORM = 3,
+    /* Default 0 (none).  The committed length the caller expects its sequences to have, in slots.  The host never
+     * reads kv_len, so where it must choose between ways of running the attention it reasons about the cache
+     * capacity S_max; a context sized for 32 k slots that serves 2 k-token sequences is better described by this
+     * hint.  It only steers that choice: any kv_len up to S_max - N stays valid. */
+    VISPEC_OPT_KV_LEN_HINT = 4,
+    /* Default 0 (1 if the environment has VISPEC_DEBUG set at context creation).  vispec_tree_verify_attn also
+     * checks its `positions` argument on the device: positions[b][i] == kv_len[b] + (set bits of tree_mask row
+     * i) - 1, the rule "position = committed length + depth" for a mask built from a parent array.  A mismatch sets
+     * the status word VISPEC_E_POSITIONS; the attention itself runs unchanged (it does not use positions).  One
+     * extra small launch per call, so off by default. */
+    VISPEC_OPT_CHECK_POSITIONS = 5
 } vispec_option;
 
 /* Set an option of the context (host call, takes effect for later calls).  Errors: E_NULL,
@@ -151,8 +168,9 @@ int vispec_tree_mask_build(vispec_ctx* ctx, const int32_t* parents, int B, int N
  * An empty A gives out = 0 and lse = -inf.  tree_mask is an INPUT (any bit pattern is honoured,
  * it is never re-derived from parents).  Cache slots at or beyond S + N are never interpreted
  * (they may hold NaN patterns); tree rows that a node's mask hides get weight exactly 0 and must
- * hold finite values, as rows written by the K/V projection do.  `positions` [B,N] (kv_len + depth) is accepted for interface
- * completeness; q and the cached k arrive already rotated, so it is not read.  It may be NULL.
+ * hold finite values, as rows written by the K/V projection do.  `positions` [B,N] (kv_len + depth) may be
+ * NULL: q and the cached k arrive already rotated (vispec_rope_tree_rows is the call that uses positions), so the
+ * attention does not need it; with VISPEC_OPT_CHECK_POSITIONS on it is checked against kv_len and tree_mask.
  * k_cache / v_cache must be the pointers registered for `layer` (or NULL to use them).
  * A sequence with kv_len[b] < 0 or kv_len[b] + N > S_max gets out = 0 and the status word
  * VISPEC_E_RANGE.  Needs a workspace (vispec_ctx_set_workspace).
@@ -335,8 +353,19 @@ int vispec_accept_commit(vispec_ctx* ctx, int layer_begin, int layer_end, const 
 
 /* Read and clear the device status word (synchronises `stream`; not a hot call).
  * `*code` (host) receives VISPEC_OK or the first asynchronous error recorded since the last poll.  When that
- * is VISPEC_E_TIMEOUT the arrival counters at the head of the workspace are zeroed on `stream` as well. */
+ * is VISPEC_E_TIMEOUT the arrival counters at the head of the workspace are zeroed on `stream` as well.
+ * out and lse of an attention call that ended in VISPEC_E_TIMEOUT are undefined (a block that gave up leaves
+ * its rows unwritten or half merged); only the status word says so. */
 int vispec_status_poll(vispec_ctx* ctx, int* code /*host*/, void* stream);
+
+/* Self-test of the bounded waits (Sec. 3.1 has no counterpart: this serves failure detection).  Every device-side
+ * wait of the attention kernels polls a barrier for a limited time and then gives up; this call runs that wait
+ * routine on a barrier nobody ever arrives on, with `limit_cycles` SM clock cycles (1 .. 2^31) as the limit, and a
+ * second waiter that must be released by the first one's give-up flag.  The kernel returns, the status word
+ * becomes VISPEC_E_TIMEOUT, and - as a call that gave up half way may - it leaves a non-zero arrival counter at the
+ * head of the workspace, which vispec_status_poll clears.  Nothing else is touched.  Needs a workspace.
+ * Host errors: E_NULL, E_RANGE (limit), E_WORKSPACE, E_CUDA. */
+int vispec_selftest_bounded_wait(vispec_ctx* ctx, long long limit_cycles, void* stream);
 
 /* Number of kernels the library has launched through this context since creation (host counter). */
 int vispec_launch_count(const vispec_ctx* ctx, uint64_t* out /*host*/);

@@ -19,7 +19,7 @@ VISPEC_OK = 0
 STATUS_NAMES = {
     0: "VISPEC_OK", -1: "VISPEC_E_NULL", -2: "VISPEC_E_ALIGN", -3: "VISPEC_E_SHAPE", -4: "VISPEC_E_RANGE",
     -5: "VISPEC_E_UNSUPPORTED", -6: "VISPEC_E_CUDA", -7: "VISPEC_E_TIMEOUT", -8: "VISPEC_E_BAD_TREE",
-    -9: "VISPEC_E_UNREGISTERED", -10: "VISPEC_E_WORKSPACE",
+    -9: "VISPEC_E_UNREGISTERED", -10: "VISPEC_E_WORKSPACE", -11: "VISPEC_E_POSITIONS",
 }
 EXPORTS = [
     "vispec_strerror", "vispec_ctx_create", "vispec_ctx_destroy", "vispec_workspace_bytes",
@@ -27,11 +27,13 @@ EXPORTS = [
     "vispec_tree_verify_attn", "vispec_accept", "vispec_kv_compact", "vispec_status_poll",
     "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows", "vispec_accept_sampled", "vispec_tree_rerank",
     "vispec_cache_register_paged", "vispec_tree_verify_attn_paged", "vispec_kv_compact_paged",
-    "vispec_accept_commit_paged", "vispec_rope_tree_rows_paged",
+    "vispec_accept_commit_paged", "vispec_rope_tree_rows_paged", "vispec_selftest_bounded_wait",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
 OPT_SPLIT_FORM = 3
+OPT_KV_LEN_HINT = 4
+OPT_CHECK_POSITIONS = 5
 
 
 class VispecShape(ctypes.Structure):
@@ -81,6 +83,7 @@ def load() -> ctypes.CDLL:
             "vispec_rope_tree_rows": [vp, ci, vp, vp, vp, vp, vp, ci, ci, cf, vp],
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
+            "vispec_selftest_bounded_wait": [vp, ctypes.c_longlong, vp],
             "vispec_tree_verify_attn_static": [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp],
         }
         for name, argtypes in sigs.items():
@@ -276,6 +279,9 @@ class VerifyContext:
         code = ctypes.c_int()
         _check(self.lib.vispec_status_poll(self.handle, ctypes.byref(code), _stream()), "vispec_status_poll")
         return code.value
+
+    def selftest_bounded_wait(self, limit_cycles: int) -> None:
+        _check(self.lib.vispec_selftest_bounded_wait(self.handle, limit_cycles, _stream()), "vispec_selftest_bounded_wait")
 
     def launch_count(self) -> int:
         n = ctypes.c_uint64()

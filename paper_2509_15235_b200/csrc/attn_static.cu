@@ -9,7 +9,7 @@
 // from module load until exit.
 #include "vispec_internal.h"
 
-// 16 MiB: room for up to 503 partial results of 64 query rows at D = 128 (33,280 bytes each)
+// 16 MiB: room for up to 502 partial results of 64 query rows at D = 128 (33,280 bytes each)
 // behind the 64 KiB header the workspace layout reserves.
 #define VISPEC_STATIC_SCRATCH_BYTES (16u << 20)
 
@@ -30,6 +30,9 @@ DeviceSetup g_setup[kMaxDevices];
 // In host code the names g_static_scratch / g_static_status are only handles for the runtime, not
 // device addresses, so they must never be handed to a kernel directly: ask the runtime where the
 // symbols live on the current device.
+// No lock: two host threads that make their first call on a device at the same moment both run the queries below
+// and store the same addresses and the same SM count, and `done` is set last, so whichever thread reads it as true
+// finds the fields filled; the worst case is that the queries run twice.
 int setup_current_device(int dev) {
     DeviceSetup& s = g_setup[dev];
     if (s.done) return VISPEC_OK;

@@ -898,10 +898,12 @@ static int tc5_cluster_size(const AttnArgs& a, int units) {
     // and second phase), the steps of the busiest CTA at 1.2 per step or at the HBM share of that many CTAs (64 KB
     // per step at 5.2 TB/s over the cluster form's CTAs, 6.6 TB/s over the even split's; the row blocks of one kv
     // head read the same tiles, so only one in n_mblocks comes from HBM), and 0.25 per partial a unit is merged
-    // from.  The host knows only the capacity S_max, not kv_len: the estimate is for full caches.
+    // from.  The host knows only the capacity S_max, not kv_len: the estimate is for full caches unless the caller
+    // has given the length it expects (VISPEC_OPT_KV_LEN_HINT).
     const int n_mblocks = pair ? 1 : (rows_total + 127) / 128;
-    const double steps = (double)((a.S_max + STEP - 1) / STEP), T = steps * units;
-    const double n_c = (double)units * best, per_c = (double)(((a.S_max + STEP - 1) / STEP + best - 1) / best);
+    const int slots = (a.kv_len_hint > 0 && a.kv_len_hint + a.N < a.S_max) ? a.kv_len_hint + a.N : a.S_max;
+    const double steps = (double)((slots + STEP - 1) / STEP), T = steps * units;
+    const double n_c = (double)units * best, per_c = (double)(((slots + STEP - 1) / STEP + best - 1) / best);
     const double est_c = 11.0 + per_c * fmax(1.2, n_c * 0.0125 / n_mblocks);
     const double n_e = fmin((double)a.sm_count, fmax(1.0, T / 2.0));
     const double est_e = 14.0 + (T / n_e) * fmax(1.2, n_e * 0.00973 / n_mblocks) + 0.25 * (n_e / units);
@@ -987,6 +989,41 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     if (err != cudaSuccess) return err;
     ++*n_launches;
     return cudaSuccess;
+}
+
+namespace {
+
+// The attention kernels' wait routine on a barrier that never completes: thread 0 runs out of its limit and raises the
+// give-up flag; thread 32 waits on a second such barrier with the ordinary (long) limit and must be released by that
+// flag.  Then the block reports VISPEC_E_TIMEOUT and leaves one arrival counter non-zero, as a call that gave up
+// between a partial's arrival and the unit's merge would.
+__global__ void __launch_bounds__(64)
+bounded_wait_selftest_kernel(long long limit, int* status, int* counters) {
+    __shared__ __align__(8) unsigned long long bars[2];
+    __shared__ int flag;
+    volatile int* abort_flag = &flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars[0]), 1);
+        mbar_init(smem_u32(&bars[1]), 1);
+        flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool gave_up = false;
+    if (threadIdx.x == 0) gave_up = !mbar_wait(smem_u32(&bars[0]), 0, abort_flag, limit);
+    if (threadIdx.x == 32) gave_up = !mbar_wait(smem_u32(&bars[1]), 0, abort_flag);
+    const int n = __syncthreads_count(gave_up);
+    if (threadIdx.x == 0 && n == 2 && *abort_flag) {
+        atomicCAS(status, 0, (int)VISPEC_E_TIMEOUT);
+        atomicAdd(counters, 1);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_bounded_wait_selftest(long long limit, int* status, int* counters, cudaStream_t st) {
+    bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(limit, status, counters);
+    return cudaGetLastError();
 }
 
 cudaError_t init_stream_probe() {

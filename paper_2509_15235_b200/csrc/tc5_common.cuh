@@ -26,9 +26,10 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait for the completion of the phase with parity `parity`.  Returns false after ~kWaitCycles
+// Bounded wait for the completion of the phase with parity `parity`.  Returns false after ~limit cycles
 // or as soon as another role has raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = kWaitCycles) {
     long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
         uint32_t ok;
@@ -42,7 +43,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+            else if (now - t0 > limit) { *abort_flag = 1; return false; }
         }
     }
 }

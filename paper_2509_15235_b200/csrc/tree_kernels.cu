@@ -334,10 +334,12 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
                  __nv_bfloat16* __restrict__ v_cache, double log2_theta, int N, int Hq, int Hkv, int D, int S_max,
                  int* status, const RowMap rmap) {
     __shared__ double cs[64], sn[64];
-    // The attention that follows may start its prologue (and stream cache rows below kv_len, which this kernel never
-    // writes) while these blocks run; it waits for this grid to finish before it reads q or a tree row.
+    // First wait for the kernel before this one (q / k_new / v_new may come from it, and so may kv_len), only then let
+    // the next kernel in: an attention call that follows reads kv_len and committed cache rows before its own wait,
+    // and must not do so while the kernel two places back (a commit, say) is still running.  Its prologue still
+    // overlaps these blocks; this kernel writes only q and slots at or above kv_len.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");       // q / k_new / v_new may come from the kernel just before
     const int i = blockIdx.x, b = blockIdx.y, half = D / 2;
     const int S = kv_len[b];
     if (S < 0 || S + N > S_max) {
@@ -379,6 +381,27 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
     if (row < Hq + Hkv) rope_rotate8(lo, hi, cs + c8, sn + c8);
     dst[c8 / 8] = lo;
     dst[(c8 + half) / 8] = hi;
+}
+
+namespace {
+// One thread per (sequence, node): the position a draft-tree node carries is the committed length plus its depth, and
+// the depth is the number of its ancestors, i.e. the set bits of its mask row minus its own.
+__global__ void check_positions_kernel(const int32_t* __restrict__ positions, const int32_t* __restrict__ kv_len,
+                                       const uint64_t* __restrict__ mask, int B, int N, int* status) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= B * N) return;
+    const int b = idx / N, W = (N + 63) >> 6;
+    int bits = 0;
+    for (int w = 0; w < W; ++w) bits += __popcll(mask[(size_t)idx * W + w]);
+    if (positions[idx] != kv_len[b] + bits - 1) record_status(status, VISPEC_E_POSITIONS);
+}
+}  // namespace
+
+cudaError_t launch_check_positions(const int32_t* positions, const int32_t* kv_len, const uint64_t* mask, int B, int N,
+                                   int* status, cudaStream_t st) {
+    if (B * N == 0) return cudaSuccess;
+    check_positions_kernel<<<(B * N + 127) / 128, 128, 0, st>>>(positions, kv_len, mask, B, N, status);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,

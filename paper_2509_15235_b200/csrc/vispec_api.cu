@@ -58,6 +58,7 @@ const char* vispec_strerror(int status) {
         case VISPEC_E_BAD_TREE: return "parent array is not a valid tree";
         case VISPEC_E_UNREGISTERED: return "layer cache not registered (or pointers differ)";
         case VISPEC_E_WORKSPACE: return "workspace missing or too small";
+        case VISPEC_E_POSITIONS: return "positions differ from kv_len + depth";
         default: return "unknown status";
     }
 }
@@ -90,6 +91,7 @@ int vispec_ctx_create(vispec_ctx** out, const vispec_shape* s, int device) {
     c->h_v.assign(s->layers, nullptr);
     const char* fg = std::getenv("VISPEC_FORCE_GENERIC");
     c->force_generic = fg && fg[0] == '1';
+    c->check_positions = std::getenv("VISPEC_DEBUG") != nullptr;
     c->k_map.resize(s->layers);
     c->page_rows.assign(s->layers, 0);
     c->num_blocks.assign(s->layers, 0);
@@ -132,6 +134,10 @@ int vispec_ctx_set_option(vispec_ctx* c, int option, int value) {
         case VISPEC_OPT_SPLIT_FORM:
             if (value < 0 || value > 3) return VISPEC_E_RANGE;
             c->tc5_path = value; return VISPEC_OK;
+        case VISPEC_OPT_KV_LEN_HINT:
+            if (value < 0) return VISPEC_E_RANGE;
+            c->kv_len_hint = value; return VISPEC_OK;
+        case VISPEC_OPT_CHECK_POSITIONS: c->check_positions = value != 0; return VISPEC_OK;
         default: return VISPEC_E_UNSUPPORTED;
     }
 }
@@ -228,7 +234,6 @@ int vispec_tree_mask_build(vispec_ctx* c, const int32_t* parents, int B, int N, 
 int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void* k_cache, const void* v_cache,
                             const int32_t* kv_len, const uint64_t* tree_mask, const int32_t* positions,
                             int B, int N, float scale, void* out, float* lse, void* stream) {
-    (void)positions;
     if (!c || !q || !kv_len || !tree_mask || !out) return VISPEC_E_NULL;
     if (!aligned(q, 16) || !aligned(out, 16)) return VISPEC_E_ALIGN;
     const vispec_shape& s = c->shape;
@@ -246,11 +251,17 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
     a.sm_count = c->sm_count;
     a.early_prefetch = c->early_prefetch;
     a.tc5_path = c->tc5_path;
+    a.kv_len_hint = c->kv_len_hint;
     a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
     int n = 0;
     cudaError_t err = (!c->force_generic && attn_tc5_supports(a)) ? launch_attn_tc5(a, (cudaStream_t)stream, &n)
                                                                   : launch_attn_generic(a, (cudaStream_t)stream, &n);
     c->launches += n;
+    if (err == cudaSuccess && c->check_positions && positions && B > 0) {
+        // after the attention, so that the attention keeps its place right behind its predecessor on the stream
+        err = launch_check_positions(positions, kv_len, tree_mask, B, N, c->d_status, (cudaStream_t)stream);
+        c->launches += 1;
+    }
     return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
 }
 
@@ -276,6 +287,7 @@ int vispec_tree_verify_attn_paged(vispec_ctx* c, int layer, const void* q, const
     a.sm_count = c->sm_count;
     a.early_prefetch = c->early_prefetch;
     a.tc5_path = c->tc5_path;
+    a.kv_len_hint = c->kv_len_hint;
     a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
     a.block_table = block_table; a.table_stride = table_stride;
     a.page_rows = c->page_rows[layer]; a.num_blocks = c->num_blocks[layer]; a.token_major = c->token_major[layer];
@@ -493,6 +505,16 @@ int vispec_status_poll(vispec_ctx* c, int* code, void* stream) {
     // a call that gave up on a wait may have left arrival counters behind: the next call finds them zero again
     if (v == VISPEC_E_TIMEOUT && c->ws && cudaMemsetAsync(c->ws, 0, kCounterBytes, st) != cudaSuccess) return VISPEC_E_CUDA;
     *code = v;
+    return VISPEC_OK;
+}
+
+int vispec_selftest_bounded_wait(vispec_ctx* c, long long limit_cycles, void* stream) {
+    if (!c) return VISPEC_E_NULL;
+    if (limit_cycles < 1 || limit_cycles > (1ll << 31)) return VISPEC_E_RANGE;
+    if (!c->ws) return VISPEC_E_WORKSPACE;
+    if (launch_bounded_wait_selftest(limit_cycles, c->d_status, (int*)c->ws, (cudaStream_t)stream) != cudaSuccess)
+        return VISPEC_E_CUDA;
+    c->launches += 1;
     return VISPEC_OK;
 }
 

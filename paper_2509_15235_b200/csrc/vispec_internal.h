@@ -24,6 +24,8 @@ struct vispec_ctx {
     bool force_generic = false;     // VISPEC_OPT_FORCE_GENERIC (or VISPEC_FORCE_GENERIC=1 at context creation)
     bool early_prefetch = true;     // VISPEC_OPT_EARLY_PREFETCH
     int tc5_path = 0;               // VISPEC_OPT_SPLIT_FORM: 0 automatic, 1 partials in global memory, 2 clusters, 3 merge kernel always
+    int kv_len_hint = 0;            // VISPEC_OPT_KV_LEN_HINT
+    bool check_positions = false;   // VISPEC_OPT_CHECK_POSITIONS (or VISPEC_DEBUG in the environment at context creation)
 };
 
 namespace vispec {
@@ -80,6 +82,7 @@ struct AttnArgs {
     int sm_count;
     bool early_prefetch;   // committed-prefix tiles may be read before the preceding kernel has completed
     int tc5_path;          // 0 automatic, 1 partials in global memory (3: merge kernel always), 2 clusters where possible
+    int kv_len_hint;       // committed length the caller expects (0: unknown, reason about S_max)
     const CUtensorMap* k_map; const CUtensorMap* v_map;
     // paged cache (page_rows != 0): pool blocks of page_rows slots, block_table [B][table_stride]; S_max is then
     // table_stride * page_rows
@@ -93,6 +96,11 @@ cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, int* n_launc
 bool attn_tc5_supports(const AttnArgs& a);
 cudaError_t init_attn_tc5();           // once per device, with that device current
 cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches);
+// The bounded wait of the attention kernels on a barrier that never completes (failure-detection self-test).
+cudaError_t launch_bounded_wait_selftest(long long limit, int* status, int* counters, cudaStream_t st);
+// positions[b][i] == kv_len[b] + popcount(mask row i) - 1, else status VISPEC_E_POSITIONS.
+cudaError_t launch_check_positions(const int32_t* positions, const int32_t* kv_len, const uint64_t* mask, int B, int N,
+                                   int* status, cudaStream_t st);
 // Streaming-read probe over the rows one attention call reads (measurement aid).
 cudaError_t init_stream_probe();
 cudaError_t launch_stream_probe(const AttnArgs& a, cudaStream_t st);

@@ -133,7 +133,7 @@ def test_large_scores_stay_finite(gu):
     mask, _, _ = oracle.tree_mask(np.arange(-1, N - 1, dtype=np.int32)[None])
     out, lse, _ = gu.run_attn(q, k, v, [150], mask, 0.125)
     want, want_lse = oracle.tree_attn(q, k, v, [150], mask, 0.125)
-    assert np.isfinite(out).all() and np.abs(out - want).max() <= 3e-2
+    assert np.isfinite(out).all() and np.abs(out - want).max() <= TOL
     assert np.abs(lse - want_lse).max() <= 2e-3 * np.abs(want_lse).max()
 
 
@@ -192,6 +192,11 @@ def test_full_size_batched_variable_length_parity(gu):
     want, want_lse = oracle.tree_attn(q[:, :, heads], k[:, heads], v[:, heads], kv_len, mask, 1 / math.sqrt(cfg.D))
     assert np.abs(out[:, :, heads] - want).max() <= TOL
     assert np.abs(lse[:, heads] - want_lse).max() <= LSE_TOL
+    # and every one of the 40 heads of the longest sequence
+    b = int(np.argmax(kv_len))
+    want, want_lse = oracle.tree_attn(q[b:b + 1], k[b:b + 1], v[b:b + 1], kv_len[b:b + 1], mask[b:b + 1], 1 / math.sqrt(cfg.D))
+    assert np.abs(out[b:b + 1] - want).max() <= TOL
+    assert np.abs(lse[b:b + 1] - want_lse).max() <= LSE_TOL
 
 
 @pytest.mark.parametrize("name", ["qwen3b_S2048_N16_B1", "qwen3b_S8192_N60_B4", "qwen3b_S32768_N128_B1",

@@ -103,3 +103,56 @@ def test_rope_rows_host_errors_and_empty_batch():
     torch.cuda.synchronize()
     assert ctx.launch_count() == before + 1 and ctx.status_poll() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (8, 2)])
+def test_commit_then_rope_then_attention_chained_on_one_stream(Hq, Hkv):
+    """The end of one cycle and the start of the next, enqueued back to back with nothing in between:
+    vispec_accept_commit writes the new kv_len and commits rows, vispec_rope_tree_rows places the next tree's rows behind
+    the new length, vispec_tree_verify_attn (early prefix reads on) takes that same device kv_len.  The attention must
+    see the committed length and rows; everything against the oracle's chain."""
+    from paper_2509_15235_b200 import binding
+    import gpu_util as gu
+    B, N, D, S_max = 2, 24, 128, 1792
+    rng = np.random.Generator(np.random.Philox(31 + Hq))
+    scale = 1.0 / np.sqrt(D)
+    for rep in range(4):
+        kv_len = np.array([1500 + 7 * rep, 901 - 3 * rep], dtype=np.int32)
+        kc = synth.normal_bf16((B, Hkv, S_max, D), 700 + rep); vc = synth.normal_bf16((B, Hkv, S_max, D), 710 + rep)
+        parents1 = np.stack([synth.draw_tree(N, 6, 4, rng) for _ in range(B)])
+        target = rng.integers(0, 50, size=(B, N)).astype(np.int32)
+        draft = np.where(rng.random((B, N)) < 0.8, np.take_along_axis(target, np.maximum(parents1, 0), 1),
+                         rng.integers(50, 99, size=(B, N))).astype(np.int32)
+        parents2 = np.stack([synth.draw_tree(N, 6, 4, rng) for _ in range(B)])
+        q2 = synth.normal_bf16((B, N, Hq, D), 720 + rep)
+        k2 = synth.normal_bf16((B, N, Hkv, D), 730 + rep); v2 = synth.normal_bf16((B, N, Hkv, D), 740 + rep)
+        # the oracle's chain
+        o_path, o_len, _ = oracle.accept(draft, target, parents1)
+        o_k, o_v, o_new = oracle.kv_compact(kc, vc, o_path, o_len, kv_len)
+        mask2, depth2, _ = oracle.tree_mask(parents2)
+        positions2 = (o_new[:, None] + depth2).astype(np.int32)
+        o_q, o_k2, o_v2, skipped = oracle.rope_rows(q2, k2, v2, positions2, o_new, o_k, o_v, 1e4)
+        assert skipped == 0
+        want, want_lse = oracle.tree_attn(o_q, o_k2, o_v2, o_new, mask2, scale)
+        # the same chain on one stream, no host involvement between the calls
+        ctx = binding.VerifyContext(B, N, Hq, Hkv, D, S_max, 1)
+        kd, vd = gu.bf16_dev(kc), gu.bf16_dev(vc)
+        ctx.cache_register(0, kd, vd)
+        qd, k2d, v2d = gu.bf16_dev(q2), gu.bf16_dev(k2), gu.bf16_dev(v2)
+        path = torch.zeros((B, N), dtype=torch.int32, device="cuda")
+        alen = torch.zeros(B, dtype=torch.int32, device="cuda"); bonus = torch.zeros_like(alen)
+        new_len = torch.zeros_like(alen)
+        out = torch.full((B, N, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((B, Hq, N), float("nan"), dtype=torch.float32, device="cuda")
+        args = (gu.i32_dev(draft), gu.i32_dev(target), gu.i32_dev(parents1), gu.i32_dev(kv_len), gu.i32_dev(positions2),
+                gu.u64_dev(mask2))
+        torch.cuda.synchronize()
+        ctx.accept_commit(0, 1, args[0], args[1], args[2], args[3], path, alen, bonus, new_len)
+        ctx.rope_tree_rows(0, qd, k2d, v2d, args[4], new_len, 1e4)
+        ctx.tree_verify_attn(0, qd, new_len, args[5], scale, out, lse)
+        torch.cuda.synchronize()
+        assert ctx.status_poll() == 0
+        assert np.array_equal(new_len.cpu().numpy(), o_new)
+        assert np.abs(out.float().cpu().numpy() - want).max() <= 2e-2
+        assert np.abs(lse.cpu().numpy() - want_lse).max() <= 2e-3
+        ctx.close()

@@ -48,12 +48,17 @@ def test_static_entry_matches_regular_entry_on_two_calls_in_a_row():
     s1, s2 = 1 / math.sqrt(128), 0.07
     got1 = _static(p1, s1)
     got2 = _static(p2, s2)                                      # runs on top of p1's leftovers
+    import oracle
     for p, s, got in ((p1, s1, got1), (p2, s2, got2)):
         want, want_lse, status = gu.run_attn(p["q"], p["k"], p["v"], p["kv_len"], p["mask"], s)
         assert status == 0 and got[2] == 0
         assert not np.isnan(got[0]).any()
         assert np.abs(got[0] - want).max() <= TOL
         assert np.abs(got[1] - want_lse).max() <= 2e-3
+        # and against the oracle itself, not only against the other entry point
+        ref, ref_lse = oracle.tree_attn(p["q"], p["k"], p["v"], p["kv_len"], p["mask"], s)
+        assert np.abs(got[0] - ref).max() <= TOL
+        assert np.abs(got[1] - ref_lse).max() <= 2e-3
 
 
 def test_static_entry_rejects_problems_beyond_its_scratch_and_bad_arguments():
