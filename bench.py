@@ -36,13 +36,19 @@ if ROOT not in sys.path:
 
 METRIC = "verify-attention KV GB/s (tree-verify step: mask + L x attention + accept + compact)"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) of one attention launch of the benchmarked workload, from the ncu
-# capture summarised under profiles/; None until a capture exists.
+# DRAM bytes (read + write) of one attention launch, per workload, from an ncu capture of that launch
+# (dram__bytes_read.sum + dram__bytes_write.sum, two launches averaged).  A figure is only valid for the kernel it was
+# taken on: set an entry to None when the attention kernel changes and take the counters again.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    "llava7b": 66_345_000,                # profiles/attn_tc5_kernel_llava7b.md: 65.58 MB read + 0.77 MB written
-    "llava13b_b4": 335_470_000,           # profiles/attn_tc5_kernel_llava13b_b4.md: 330.22 MB read + 5.25 MB written
-    "qwen3b_S32768_N16_B8": 274_550_000,  # profiles/attn_tc5_kernel_qwen3b_S32768_N16_B8.md (merge kernel adds 9.6 MB)
+    "llava7b": 66_345_000,                # 65.58 MB read + 0.77 MB written
+    "llava13b_b4": 335_470_000,           # 330.22 MB read + 5.25 MB written
+    "qwen3b_S32768_N16_B8": 274_550_000,  # attention launch only; the merge kernel adds 9.6 MB
 }
+FALLBACK_BF16_TFLOPS = 1400.0             # sustained figure of the fallback measurement
+EXP_PER_CLK_PER_SM = 16                   # special-function lanes of one SM (4 per scheduler)
+# Workloads timed briefly after the headline (attention sweep only), each against its own binding roofline.
+OTHER_WORKLOADS = [("qwen7b", 28, False), ("llava13b_b4", 8, False), ("qwen3b_S8192_N16_B4", 16, False),
+                   ("qwen3b_S8192_N60_B4", 16, False), ("llava7b", 8, True)]
 
 
 def parse_args():
@@ -56,6 +62,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     ap.add_argument("--split-form", type=int, default=0, help="VISPEC_OPT_SPLIT_FORM of the context (0 automatic; see vispec.h)")
+    ap.add_argument("--no-others", action="store_true", help="skip the short timed runs of the other workloads")
     ap.add_argument("--no-sampled", action="store_true", help="skip the timing of vispec_accept_sampled")
     ap.add_argument("--paged", type=int, default=0, help="serve the caches from a block pool of this many slots per block (16/32/64/128)")
     ap.add_argument("--token-major", action="store_true", help="with --paged: pool blocks are [slots, kv heads, D] instead of [kv heads, slots, D]")
@@ -65,12 +72,40 @@ def parse_args():
 
 
 def measured_peaks():
+    """(HBM GB/s, sustained bf16 TFLOP/s, max SM MHz, "measured" | "fallback")."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         with open(p) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return FALLBACK_HBM_GBS, "fallback"
+        return (float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", FALLBACK_BF16_TFLOPS)),
+                float(d.get("sm_max_mhz", 1965.0)), "measured")
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, 1965.0, "fallback"
+
+
+def attention_roofline(cfg, kv_len, us_per_launch, sm_count, traffic=None):
+    """The roofline of one attention launch: the time each resource needs for the launch's algorithmic work - K and V
+    rows from HBM (512 B per cached token per kv head at D = 128), the two contractions on the tensor cores
+    (4*D*G*N flops per cached token per kv head, against the sustained bf16 figure: the launch sits inside a long
+    step) and the softmax's exponentials on the special-function units (G*N per cached token per kv head) - names
+    the largest as the bound and reports the achieved rate against that resource's peak."""
+    hbm_gbs, tflops, sm_mhz, kind = measured_peaks()
+    tokens = int(sum(int(s) + cfg.N for s in kv_len)) * cfg.Hkv          # cached tokens x kv heads
+    kv_bytes = tokens * 4 * cfg.D
+    flops = tokens * 4 * cfg.D * cfg.G * cfg.N
+    exps = tokens * cfg.G * cfg.N
+    exp_peak = EXP_PER_CLK_PER_SM * sm_count * sm_mhz * 1e6               # exponentials per second
+    t = {"hbm": kv_bytes / (hbm_gbs * 1e9), "tensor": flops / (tflops * 1e12), "alu": exps / exp_peak}
+    bound = max(t, key=t.get)
+    sec = us_per_launch * 1e-6
+    if bound == "hbm":
+        achieved, peak, unit = kv_bytes / sec / 1e9, hbm_gbs, "GB/s"
+    elif bound == "tensor":
+        achieved, peak, unit = flops / sec / 1e12, tflops, "TFLOP/s"
+    else:
+        achieved, peak, unit = exps / sec / 1e12, exp_peak / 1e12, "Texp/s"
+    return {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+            "peak_kind": f"of {kind}", "floor_us": {k: v * 1e6 for k, v in t.items()},
+            "kv_gbs": kv_bytes / sec / 1e9, "pct_of_8TBs": 100.0 * kv_bytes / sec / 8e12, "traffic": traffic}
 
 
 # ------------------------------------------------------------------------------------ rank logic
@@ -111,7 +146,7 @@ class ClockSampler:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -361,6 +396,79 @@ class HostStep:
         self.s_out.synchronize()
 
 
+def time_other_workload(name, layers, redundant, device, min_seconds=0.4):
+    """Attention sweep of one further workload (L layers, each its own cache pair, graph replay), timed for at least
+    `min_seconds` with the clocks sampled meanwhile, against that workload's own binding roofline.  Trees and
+    lengths come from the seeded generators; q/K/V are N(0,1) bf16 drawn on the device (timing only: these
+    workloads have their parity tests).  `redundant`: the image span of every head repeats one key (Sec. 4.1, Eq. 2)."""
+    import torch
+    from paper_2509_15235_b200 import binding, synth
+    cfg = synth.get_config(name)
+    tree = synth.make_tree_inputs(cfg)
+    dev = torch.device("cuda", device)
+    L = min(layers, cfg.layers)
+    B, N, Hq, Hkv, D = cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.D
+    ctx = binding.VerifyContext(B, N, Hq, Hkv, D, cfg.S_max, L, device=device)
+    g = torch.Generator(device=dev).manual_seed(cfg.config_id)
+    ks, vs = [], []
+    for l in range(L):
+        k = torch.randn((B, Hkv, cfg.S_max, D), generator=g, device=dev, dtype=torch.bfloat16)
+        v = torch.randn((B, Hkv, cfg.S_max, D), generator=g, device=dev, dtype=torch.bfloat16)
+        if redundant:
+            k[:, :, :cfg.n_image] = k[:, :, :1]
+        ctx.cache_register(l, k, v)
+        ks.append(k); vs.append(v)
+    q = torch.randn((L, B, N, Hq, D), generator=g, device=dev, dtype=torch.bfloat16)
+    out = torch.empty_like(q)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    kv_len, parents = i32(tree["kv_len"]), i32(tree["parents"])
+    mask = torch.zeros((B, N, (N + 63) // 64), dtype=torch.int64, device=dev)
+    ctx.tree_mask_build(parents, mask)
+    scale = 1.0 / math.sqrt(D)
+
+    def sweep():
+        for l in range(L):
+            ctx.tree_verify_attn(l, q[l], kv_len, mask, scale, out[l])
+
+    n0 = ctx.launch_count()
+    sweep()
+    torch.cuda.synchronize()
+    launches_per_call = (ctx.launch_count() - n0) // L
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        sweep()
+    for _ in range(5):
+        graph.replay()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device)
+    sampler.start()
+    time.sleep(0.15)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps, ms = 0, 0.0
+    while ms < min_seconds * 1e3:
+        chunk = max(20, reps)
+        e0.record()
+        for _ in range(chunk):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms += e0.elapsed_time(e1)
+        reps += chunk
+    clocks = sampler.stop()
+    status = ctx.status_poll()
+    us = ms * 1e3 / (reps * L)
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    res = attention_roofline(cfg, tree["kv_len"], us, sm_count, NCU_TRAFFIC_BYTES_PER_LAUNCH.get(name) if not redundant else None)
+    res.update({"workload": name + ("+redundant_image_keys" if redundant else ""), "layers": L, "us_per_layer": us,
+                "sweeps": reps, "launches_per_call": launches_per_call, "status_word": status,
+                "kv_mb_per_layer": cfg.kv_bytes_per_layer(tree["kv_len"]) / 1e6,
+                "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "power_w_max")}})
+    ctx.close()
+    del ks, vs, q, out
+    torch.cuda.empty_cache()
+    return res
+
+
 # ------------------------------------------------------------------------------------ oracle legs
 
 def oracle_sample(cfg, tree, layers, budget_heads):
@@ -475,10 +583,29 @@ def main():
     ms_total = e0.elapsed_time(e1)
     attn_ms = sum(a.elapsed_time(b) for a, b in evs)
     launches = launches_per_step * args.steps
+    # The roofline figure: at least max(steps, 100) further attention sweeps (the L attention calls of a step, graph
+    # replay, events on the launching stream) and at least half a second of them, so that the clock sampler sees the
+    # load.  `value` and `ms_per_step` stay on the `steps` whole steps timed above.
+    sweep_reps, sweep_ms = 0, 0.0
+    if not args.no_graph:
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        while sweep_reps < max(args.steps, 100) or sweep_ms < 500.0:
+            chunk = max(args.steps, 100)
+            r0.record()
+            for _ in range(chunk):
+                wl.graphs[1].replay()
+            r1.record()
+            torch.cuda.synchronize()
+            sweep_ms += r0.elapsed_time(r1)
+            sweep_reps += chunk
+        launches += sweep_reps * (launches_per_step - 2)
+    barrier()
     clocks = sampler.stop() if rank == 0 else None
     status = wl.ctx.status_poll()
+    if sweep_reps == 0:
+        sweep_reps, sweep_ms = args.steps, attn_ms
 
-    ms_total, attn_ms = max_over_ranks([ms_total, attn_ms], world, "cuda")
+    ms_total, attn_ms = max_over_ranks([ms_total, attn_ms], world, "cuda")   # (the roofline sweep is rank 0's own)
     kv_bytes_step = wl.kv_bytes_per_layer * L
     value = whole_job_gbs(kv_bytes_step, args.steps, ms_total * 1e-3, world)
 
@@ -585,9 +712,16 @@ def main():
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peaks()
-    attn_s = attn_ms * 1e-3 / (args.steps * L)
-    achieved = wl.kv_bytes_per_layer / attn_s / 1e9
+    attn_s = attn_ms * 1e-3 / (args.steps * L)               # inside the timed steps
+    sweep_us = sweep_ms * 1e3 / (sweep_reps * L)             # the longer attention-only run the roofline is quoted on
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+    roof = attention_roofline(cfg, tree["kv_len"], sweep_us, sm_count,
+                              NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name) if not (args.paged or args.with_rope) else None)
+    roof.update({"kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L - int(args.with_rope)} kernel launch(es) per call)",
+                 "us_per_launch": sweep_us, "sweeps": sweep_reps})
+    others = None
+    if not args.no_others and not (args.paged or args.with_rope or args.layers):
+        others = [time_other_workload(n, l, r, local) for n, l, r in OTHER_WORKLOADS if not (n == cfg.name and not r)]
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -601,13 +735,12 @@ def main():
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
         "attn_us_per_layer": attn_s * 1e6,
-        "pct_of_8TBs": 100.0 * achieved / 8000.0,
+        "pct_of_8TBs": roof["pct_of_8TBs"],
         "read_probe": read_probe,
         "around_the_forward": sampled,
         "status_word": status,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L - int(args.with_rope)} kernel launch(es) per call)",
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)},
+        "roofline": roof,
+        "other_workloads": others,
         "clocks": clocks,
         "gpu_launches": int(launches),
     }
