@@ -69,6 +69,7 @@ def parse_args():
     ap.add_argument("--paged", type=int, default=0, help="serve the caches from a block pool of this many slots per block (16/32/64/128)")
     ap.add_argument("--token-major", action="store_true", help="with --paged: pool blocks are [slots, kv heads, D] instead of [kv heads, slots, D]")
     ap.add_argument("--with-rope", action="store_true", help="also run vispec_rope_tree_rows before each layer's attention")
+    ap.add_argument("--fused-rope", action="store_true", help="with --with-rope: one table per step and vispec_tree_verify_attn_rope per layer instead of two calls")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from Python instead of replaying graphs")
     return ap.parse_args()
 
@@ -242,6 +243,8 @@ class DeviceWorkload:
         self.positions = (self.kv_len[:, None] + self.depth).to(torch.int32).contiguous()
         self.theta = theta
         self.with_rope = True
+        self.fused_rope = False
+        self.rope_table = self.ctx.rope_table_build(self.positions, theta)
 
     def enable_paging(self, page_rows, token_major=False):
         """Re-home every layer's cache in a block pool [num_blocks, Hkv, page_rows, D] with the blocks in a seeded
@@ -265,9 +268,15 @@ class DeviceWorkload:
 
     def _pre(self):
         self.ctx.tree_mask_build(self.parents, self.mask, self.depth)
+        if self.with_rope and getattr(self, "fused_rope", False):
+            self.ctx.rope_table_build(self.positions, self.theta, self.rope_table)      # once per cycle, for every layer
 
     def _attn(self):
         for l in range(self.L):
+            if self.with_rope and self.fused_rope and not self.page_rows:
+                self.ctx.tree_verify_attn_rope(l, self.q[l], self.k_new[l], self.v_new[l], self.rope_table, self.kv_len,
+                                               self.mask, self.scale, self.out[l])
+                continue
             if self.with_rope and self.page_rows:
                 self.ctx.rope_tree_rows_paged(l, self.q[l], self.k_new[l], self.v_new[l], self.positions, self.kv_len,
                                               self.block_table, self.theta)
@@ -553,6 +562,7 @@ def main():
         wl.enable_paging(args.paged, args.token_major)
     if args.with_rope:
         wl.enable_rope(tree, 1e6 if cfg.name.startswith("qwen") else 1e4)
+        wl.fused_rope = bool(args.fused_rope)
 
     def barrier():
         if world > 1:
@@ -719,7 +729,7 @@ def main():
     sm_count = torch.cuda.get_device_properties(local).multi_processor_count
     roof = attention_roofline(cfg, tree["kv_len"], sweep_us, sm_count,
                               NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name) if not (args.paged or args.with_rope) else None)
-    roof.update({"kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2) // L - int(args.with_rope)} kernel launch(es) per call)",
+    roof.update({"kernel": f"vispec_tree_verify_attn ({(launches_per_step - 2 - int(args.with_rope and args.fused_rope)) // L - int(args.with_rope and not args.fused_rope)} kernel launch(es) per call)",
                  "us_per_launch": sweep_us, "sweeps": sweep_reps})
     others = None
     if not args.no_others and not (args.paged or args.with_rope or args.layers):
@@ -733,7 +743,7 @@ def main():
                    "kv_bytes_per_layer": wl.kv_bytes_per_layer,
                    "l2": f"inputs larger than L2: {L} layers x {wl.kv_bytes_per_layer / 1e6:.1f} MB rotate, no flush",
                    "launch": "plain C-ABI calls" if args.no_graph else "C-ABI calls captured once, replayed as 3 CUDA graphs per step",
-                   "rope_tree_rows": bool(args.with_rope), "paged_block_rows": args.paged, "paged_token_major": bool(args.token_major),
+                   "rope_tree_rows": bool(args.with_rope), "rope_fused": bool(args.with_rope and args.fused_rope), "paged_block_rows": args.paged, "paged_token_major": bool(args.token_major),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_steps_per_s": world * args.steps / (ms_total * 1e-3),
         "attn_us_per_layer": attn_s * 1e6,

@@ -180,6 +180,33 @@ int vispec_tree_verify_attn(vispec_ctx* ctx, int layer, const void* q, const voi
                             const int32_t* positions, int B, int N, float scale, void* out,
                             float* lse, void* stream);
 
+/* The angle table of the fused call below (Sec. 3.2: the target LLM, and with it its rotary position embedding, is
+ * unchanged).  For sequence b, node i, j < D/2:  angle = positions[b][i] * theta^(-2j/D), formed in fp64;
+ * `table` (DEVICE, 16-byte aligned, vispec_rope_table_bytes() bytes, caller-owned) receives B*N*D/2 (cos, sin) pairs
+ * in fp64 followed by the same pairs rounded to fp32.  positions and theta mean what they mean for
+ * vispec_rope_tree_rows.  One small launch; the table serves every layer of the cycle (positions do not depend on
+ * the layer).  Host errors: E_NULL, E_ALIGN, E_SHAPE (B, N, theta <= 1), E_CUDA. */
+int vispec_rope_table_build(vispec_ctx* ctx, const int32_t* positions, int B, int N, float theta, void* table,
+                            void* stream);
+/* Bytes of a table for B sequences of N nodes at the context's head size (host call). */
+int vispec_rope_table_bytes(const vispec_ctx* ctx, int B, int N, size_t* out /*host*/);
+
+/* vispec_rope_tree_rows followed by vispec_tree_verify_attn as one call (Sec. 3.2; Eq. 1), for contiguous caches at
+ * D = 128, at most 32 sequences and scale > 0 (anything else: VISPEC_E_UNSUPPORTED, use the two calls).  q [B,N,Hq,D]
+ * arrives UNROTATED and is not modified.  k_new, v_new [B,N,Hkv,D] are the tree's rows: k rotated in fp64 with one
+ * rounding to bf16, v copied, both written to slots kv_len[b] + i of the registered caches exactly as
+ * vispec_rope_tree_rows writes them.  Short calls (the form with one thread-block cluster per head) run as ONE
+ * launch: every thread block rotates the q rows it needs on their way into shared memory (fp32 arithmetic from the
+ * table's fp32 half; the rotated q is consumed by the score product only), and the blocks whose share of the cache
+ * contains the tree's slots write those rows before they read them.  Long calls (work split evenly over the SMs)
+ * run as two launches - the rotation kernel fed from the table, writing the rotated q into a scratch copy at the end
+ * of the workspace, then the plain attention - because there the in-kernel rotation costs more than it saves.  Everything else (tree_mask, kv_len, out, lse,
+ * status word, early prefix reads) as in vispec_tree_verify_attn; rope_table comes from vispec_rope_table_build
+ * with the same B and N.  Host errors: those of vispec_tree_verify_attn, plus E_ALIGN for k_new / v_new / table. */
+int vispec_tree_verify_attn_rope(vispec_ctx* ctx, int layer, const void* q, const void* k_new, const void* v_new,
+                                 const void* rope_table, const int32_t* kv_len, const uint64_t* tree_mask, int B, int N,
+                                 float scale, void* out, float* lse, void* stream);
+
 /* Attention without any allocation (the paper has no counterpart: this entry point exists for
  * deployment, not for the method).  It is for callers that cannot obtain device memory when they
  * need to run: a serving process whose memory pool is fixed at start-up, a plugin that receives

@@ -28,6 +28,7 @@ EXPORTS = [
     "vispec_launch_count", "vispec_tree_verify_attn_static", "vispec_ctx_set_option", "vispec_accept_commit", "vispec_stream_probe", "vispec_rope_tree_rows", "vispec_accept_sampled", "vispec_tree_rerank",
     "vispec_cache_register_paged", "vispec_tree_verify_attn_paged", "vispec_kv_compact_paged",
     "vispec_accept_commit_paged", "vispec_rope_tree_rows_paged", "vispec_selftest_bounded_wait",
+    "vispec_rope_table_build", "vispec_rope_table_bytes", "vispec_tree_verify_attn_rope",
 ]
 OPT_EARLY_PREFETCH = 1
 OPT_FORCE_GENERIC = 2
@@ -84,6 +85,9 @@ def load() -> ctypes.CDLL:
             "vispec_status_poll": [vp, ctypes.POINTER(ci), vp],
             "vispec_launch_count": [vp, ctypes.POINTER(ctypes.c_uint64)],
             "vispec_selftest_bounded_wait": [vp, ctypes.c_longlong, vp],
+            "vispec_rope_table_build": [vp, vp, ci, ci, cf, vp, vp],
+            "vispec_rope_table_bytes": [vp, ci, ci, ctypes.POINTER(ctypes.c_size_t)],
+            "vispec_tree_verify_attn_rope": [vp, ci, vp, vp, vp, vp, vp, vp, ci, ci, cf, vp, vp, vp],
             "vispec_tree_verify_attn_static": [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp],
         }
         for name, argtypes in sigs.items():
@@ -269,6 +273,25 @@ class VerifyContext:
         _check(self.lib.vispec_rope_tree_rows(self.handle, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(positions),
                                               _ptr(kv_len), B, N, ctypes.c_float(theta), _stream()),
                "vispec_rope_tree_rows")
+
+    def rope_table_build(self, positions: torch.Tensor, theta: float, table: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """vispec_rope_table_build; allocates the table (a uint8 tensor of vispec_rope_table_bytes) unless one is given."""
+        B, N = positions.shape
+        if table is None:
+            n = ctypes.c_size_t()
+            _check(self.lib.vispec_rope_table_bytes(self.handle, B, N, ctypes.byref(n)), "vispec_rope_table_bytes")
+            table = torch.empty(max(n.value, 16), dtype=torch.uint8, device=self.device)
+        _check(self.lib.vispec_rope_table_build(self.handle, _ptr(positions), B, N, ctypes.c_float(theta), _ptr(table),
+                                                _stream()), "vispec_rope_table_build")
+        return table
+
+    def tree_verify_attn_rope(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                              rope_table: torch.Tensor, kv_len: torch.Tensor, tree_mask: torch.Tensor, scale: float,
+                              out: torch.Tensor, lse: Optional[torch.Tensor] = None) -> None:
+        B, N = q.shape[0], q.shape[1]
+        _check(self.lib.vispec_tree_verify_attn_rope(self.handle, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(rope_table),
+                                                     _ptr(kv_len), _ptr(tree_mask), B, N, ctypes.c_float(scale), _ptr(out),
+                                                     _ptr(lse), _stream()), "vispec_tree_verify_attn_rope")
 
     def stream_probe(self, layer: int, kv_len: torch.Tensor, N: int) -> None:
         _check(self.lib.vispec_stream_probe(self.handle, layer, _ptr(kv_len), kv_len.shape[0], N, _stream()),

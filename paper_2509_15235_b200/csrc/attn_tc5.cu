@@ -84,7 +84,7 @@ enum { B_KFULL = 0, B_KEMPTY = B_KFULL + NSK, B_VFULL = B_KEMPTY + NSK, B_VEMPTY
        B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2,
        B_QFULL = B_PVDONE + 2, B_PAIRX = B_QFULL + 1, B_XCH = B_PAIRX + 4, B_XFREE = B_XCH + 1,
        B_SEGSYNC = B_XFREE + 1, B_COUNT = B_SEGSYNC + 1 };
-static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block too small");
+static_assert(B_COUNT * 8 + 20 <= BAR_BYTES, "barrier block too small");
 
 constexpr int SMEM_TABRING = SMEM_SCHED + ((int)sizeof(Sched) + 15) / 16 * 16;   // 8 steps x 8 block numbers (paged cache)
 constexpr int SMEM_TOTAL = SMEM_TABRING + 256;
@@ -172,12 +172,97 @@ __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensor
     return (uint32_t)t | fail | (waited ? 1u << 30 : 0u);
 }
 
+// ---- fused rotary embedding ---------------------------------------------------------------------------
+// Bounded wait of the producer until `want` softmax threads have put their share of the tree rows into the cache
+// (each counts itself in shared memory once per segment that has tree rows).
+__device__ __forceinline__ bool rows_placed(volatile int* rows_done, int want, volatile int* abort_flag) {
+    long long t0 = 0;
+    for (uint32_t it = 0; *rows_done < want; ++it) {
+        if ((it & 63) == 63) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+        }
+    }
+    return true;
+}
+// Eight pairs (x = element j of the lower half, y = element j + D/2) rotated by their angles: fp64 with one rounding
+// to bf16 for the k rows that go to the cache, fp32 for q rows (consumed by the product, never stored).
+__device__ __forceinline__ void rope8_f64(uint4& lo, uint4& hi, const double2* cs) {
+    __nv_bfloat16* a = reinterpret_cast<__nv_bfloat16*>(&lo);
+    __nv_bfloat16* b = reinterpret_cast<__nv_bfloat16*>(&hi);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const double x = (double)__bfloat162float(a[t]), y = (double)__bfloat162float(b[t]);
+        a[t] = __double2bfloat16(x * cs[t].x - y * cs[t].y);
+        b[t] = __double2bfloat16(y * cs[t].x + x * cs[t].y);
+    }
+}
+__device__ __forceinline__ void rope8_f32(uint4& lo, uint4& hi, const float2* cs) {
+    __nv_bfloat16* a = reinterpret_cast<__nv_bfloat16*>(&lo);
+    __nv_bfloat16* b = reinterpret_cast<__nv_bfloat16*>(&hi);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const float x = __bfloat162float(a[t]), y = __bfloat162float(b[t]);
+        a[t] = __float2bfloat16_rn(x * cs[t].x - y * cs[t].y);
+        b[t] = __float2bfloat16_rn(y * cs[t].x + x * cs[t].y);
+    }
+}
+// The tree rows of (sequence b, kv head kvh) with tree index in [t_lo, t_hi): k rotated, v copied, written to slots
+// S + t of the cache.  Run by the kSmx softmax threads (thread st) of the CTA whose steps contain those slots, right
+// after the Q tile; every load of a pass is issued before the first use.  Not inlined: its registers stay out of the
+// step loop's budget.
+__device__ __noinline__ void place_tree_rows(const RopeArgs p, int N_, int Hkv_, int S_max_, int b, int kvh, int S, int t_lo,
+                                             int t_hi, int st) {
+    const size_t cache_row0 = ((size_t)b * Hkv_ + kvh) * S_max_ + S;
+    const int nk = (t_hi - t_lo) * 8;             // k: one item = (row, pair of 16-byte chunks c and c + 8)
+    const int nv = (t_hi - t_lo) * 16;            // v: 16 chunks per row, copied
+    for (int i0 = st, j0 = st; i0 < nk || j0 < nv; i0 += kSmx * 2, j0 += kSmx * 4) {
+        uint4 lo[2], hi[2], x[4];
+        double2 cs[2][8];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + kSmx * u;
+            if (i < nk) {
+                const int t = t_lo + (i >> 3), c = i & 7;
+                const uint4* src = reinterpret_cast<const uint4*>(p.k_new + (((size_t)b * N_ + t) * Hkv_ + kvh) * D);
+                lo[u] = src[c]; hi[u] = src[c + 8];
+                const double2* tab = p.rope_k + ((size_t)b * N_ + t) * (D / 2) + 8 * c;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) cs[u][j] = tab[j];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = j0 + kSmx * u;
+            if (i < nv) x[u] = reinterpret_cast<const uint4*>(p.v_new + (((size_t)b * N_ + t_lo + (i >> 4)) * Hkv_ + kvh) * D)[i & 15];
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + kSmx * u;
+            if (i < nk) {
+                const int t = t_lo + (i >> 3), c = i & 7;
+                rope8_f64(lo[u], hi[u], cs[u]);
+                uint4* dst = reinterpret_cast<uint4*>(p.k_cache + (cache_row0 + t) * D);
+                dst[c] = lo[u]; dst[c + 8] = hi[u];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = j0 + kSmx * u;
+            if (i < nv) reinterpret_cast<uint4*>(p.v_cache + (cache_row0 + t_lo + (i >> 4)) * D)[i & 15] = x[u];
+        }
+    }
+}
+
 // PAGED instantiations carry the paged producer; the others are compiled without it (its call sites cost the
 // contiguous kernels registers they do not have to spare).
-template <bool PAIR, bool CL, bool PAGED>
+template <bool PAIR, bool CL, bool PAGED, bool ROPE = false>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const Tc5Params p,
-                const PagedArgs pa) {
+                const std::conditional_t<ROPE, RopeArgs, PagedArgs> pa) {
+    static_assert(!(ROPE && PAGED), "the fused rotary embedding serves contiguous caches");
     constexpr int ROWS = PAIR ? 64 : 128;      // distinct query rows per CTA
     constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
     extern __shared__ __align__(1024) unsigned char sm[];
@@ -195,6 +280,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + SMEM_BAR + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SMEM_BAR + B_COUNT * 8 + 8);
     volatile int* seg_flag = abort_flag + 1;               // this CTA delivered the last partial of the unit just finished
+    volatile int* rows_done = abort_flag + 2;              // fused rotary embedding: segments whose tree rows are in the cache
     Sched& sched = *reinterpret_cast<Sched*>(sm + SMEM_SCHED);
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
@@ -215,6 +301,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         mbar_init(bar(B_XCH), 128); mbar_init(bar(B_XFREE), 128);
         mbar_init(bar(B_SEGSYNC), kSmx);
         *abort_flag = 0;
+        *rows_done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -246,8 +333,9 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         const int unit = cta / ck, b = unit / upb, uib = unit - b * upb;
         cl_seg.b = b; cl_seg.kvh = uib / p.n_mblocks; cl_seg.mblock = uib - cl_seg.kvh * p.n_mblocks;
         cl_seg.steps = sched.steps[b]; cl_seg.S = sched.len[b];
-        cl_seg.st0 = (cr * cl_seg.steps) / ck;
-        cl_seg.n = ((cr + 1) * cl_seg.steps) / ck - cl_seg.st0;
+        // (with the fused rotary embedding the last rank also places the tree rows: the short shares go to the end)
+        cl_seg.st0 = ROPE ? (cr * cl_seg.steps + ck - 1) / ck : (cr * cl_seg.steps) / ck;
+        cl_seg.n = (ROPE ? ((cr + 1) * cl_seg.steps + ck - 1) / ck : ((cr + 1) * cl_seg.steps) / ck) - cl_seg.st0;
         cl_seg.slot = -1;
     }
     auto make_iter = [&]() {
@@ -274,11 +362,17 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     waited = (r >> 30) & 1u;
                 }
             }
+            int nseg = 0;                        // segments with tree rows met so far
             while (!PAGED && ok && si.next(sg)) {
                 const int bh = sg.b * p.Hkv + sg.kvh;
+                bool seg_counted = false;
                 for (int t = 0; t < sg.n; ++t, ++it) {
                     const int tok = (sg.st0 + t) * STEP;
                     if (!waited && tok + STEP > sg.S) { pdl_wait(); waited = true; }   // the tree's rows come from the preceding kernel
+                    if (ROPE && tok + STEP > sg.S) {
+                        if (!seg_counted) { ++nseg; seg_counted = true; }      // this segment has tree rows
+                        if (!rows_placed(rows_done, nseg * kSmx, abort_flag)) { ok = false; break; }
+                    }
                     const int sk = it % NSK, sv = it % NSV;
                     if (!mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(bar(B_KFULL + sk), STAGE_BYTES);
@@ -395,6 +489,44 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 // the tile doubles as the exchange area of the previous segment's epilogue
                 if (!mbar_wait_warp(bar(B_XFREE), (seg - 1) & 1, abort_flag)) return false;
             }
+            if constexpr (ROPE) {
+                // rotated on the way in: a thread takes the chunk pair (c, c + 8) of rows st/8, st/8 + 32, ... with its
+                // eight angles; all loads are issued before the first use
+                constexpr int PITEMS = ROWS * 8 / kSmx;
+                const int c = st & 7;
+                uint4 lo[PITEMS], hi[PITEMS];
+                float4 tab[PITEMS][4];
+#pragma unroll
+                for (int k = 0; k < PITEMS; ++k) {
+                    const int row = sg.mblock * 128 + (st >> 3) + 32 * k;
+                    lo[k] = make_uint4(0, 0, 0, 0); hi[k] = lo[k];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) tab[k][j] = make_float4(1.f, 0.f, 1.f, 0.f);
+                    if (row < rows_total) {
+                        const int node = row / G, head = sg.kvh * G + row % G;
+                        const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)sg.b * N + node) * p.Hq + head) * D);
+                        lo[k] = src[c]; hi[k] = src[c + 8];
+                        const float4* t4 = reinterpret_cast<const float4*>(pa.rope_q + ((size_t)sg.b * N + node) * (D / 2) + 8 * c);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) tab[k][j] = t4[j];
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < PITEMS; ++k) {
+                    const int r = (st >> 3) + 32 * k;
+                    rope8_f32(lo[k], hi[k], reinterpret_cast<const float2*>(tab[k]));
+                    unsigned char* dst = sm + SMEM_Q + r * 128 + ((c ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4*>(dst) = lo[k];
+                    *reinterpret_cast<uint4*>(dst + HALF_BYTES) = hi[k];
+                    if (PAIR) {
+                        *reinterpret_cast<uint4*>(dst + 64 * 128) = lo[k];
+                        *reinterpret_cast<uint4*>(dst + HALF_BYTES + 64 * 128) = hi[k];
+                    }
+                }
+                fence_async_smem();
+                mbar_arrive(bar(B_QFULL));
+                return true;
+            }
             constexpr int ITEMS = ROWS * 16 / kSmx;
             const int qc = st & 15;
             uint4 v[ITEMS];
@@ -435,6 +567,28 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             while (ok && si.next(sg)) {
                 // every S product of the previous segment has been consumed by now, so Q may be replaced
                 if (!load_q(sg, seg)) { ok = false; break; }
+                if constexpr (ROPE) {
+                    // The tree rows that this CTA's own steps will read, of all its segments at once (the producer runs
+                    // segments ahead): into the cache now, while the first tiles are on their way.  The producer holds
+                    // the tiles that contain them back until every softmax thread has counted itself in, once per such
+                    // segment.
+                    if (seg == 0) {
+                        SegIter sj = make_iter();
+                        Seg sh;
+                        int placed = 0;
+                        while (sj.next(sh)) {
+                            const int t_lo = max(0, sh.st0 * STEP - sh.S), t_hi = min(N, (sh.st0 + sh.n) * STEP - sh.S);
+                            if (t_hi <= t_lo) continue;
+                            place_tree_rows(pa, N, p.Hkv, p.S_max, sh.b, sh.kvh, sh.S, t_lo, t_hi, st);
+                            ++placed;
+                        }
+                        if (placed > 0) {
+                            __threadfence();                                          // the rows are in global memory ...
+                            asm volatile("fence.proxy.async.global;" ::: "memory");   // ... and ordered before the bulk copies that read them
+                            atomicAdd(const_cast<int*>(rows_done), placed);
+                        }
+                    }
+                }
 
                 const int row = sg.mblock * 128 + lrow;          // query row within the kv head's G*N rows
                 const bool row_ok = row < rows_total;
@@ -931,12 +1085,24 @@ cudaError_t init_attn_tc5() {
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
         if (e != cudaSuccess) return e;
     }
+    const void* rope_kernels[4] = {(const void*)attn_tc5_kernel<true, false, false, true>, (const void*)attn_tc5_kernel<false, false, false, true>,
+                                   (const void*)attn_tc5_kernel<true, true, false, true>, (const void*)attn_tc5_kernel<false, true, false, true>};
+    for (const void* k : rope_kernels) {
+        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+    }
     for (int k = 1; k <= 8; ++k) { g_max_clusters[0][k] = query_max_clusters(false, k); g_max_clusters[1][k] = query_max_clusters(true, k); }
     if (getenv("VISPEC_DEBUG")) for (int k = 1; k <= 8; ++k) fprintf(stderr, "vispec: cluster size %d: %d (rows > 64) / %d (rows <= 64) co-resident clusters\n", k, g_max_clusters[0][k], g_max_clusters[1][k]);
     // The merge blocks must be able to join an SM that an attention CTA has configured for maximum shared memory.
     e = cudaFuncSetAttribute(attn_tc5_merge_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(attn_tc5_merge_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+}
+
+bool attn_tc5_uses_clusters(const AttnArgs& a) {
+    const int rows_total = (a.Hq / a.Hkv) * a.N;
+    const int n_mblocks = rows_total <= 64 ? 1 : (rows_total + 127) / 128;
+    return tc5_cluster_size(a, a.B * a.Hkv * n_mblocks) > 0;
 }
 
 cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches) {
@@ -971,6 +1137,26 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     auto launch_attn = [&](auto kernel, int cluster) {
         return launch_pdl(kernel, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, cluster, *a.k_map, *a.v_map, p, pa);
     };
+    if (a.rope_table) {
+        // fused rotary embedding (contiguous caches): the table holds B*N*D/2 fp64 (cos, sin) pairs, then the same in fp32
+        const size_t n = (size_t)a.B * a.N * (D / 2);
+        const RopeArgs ra = {(const double2*)a.rope_table, (const float2*)((const double2*)a.rope_table + n),
+                             (const __nv_bfloat16*)a.k_new, (const __nv_bfloat16*)a.v_new, (__nv_bfloat16*)a.k, (__nv_bfloat16*)a.v,
+                             own_merge ? (int*)a.ws : nullptr};
+        auto launch_rope = [&](auto kernel, int cluster) {
+            return launch_pdl(kernel, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, cluster, *a.k_map, *a.v_map, p, ra);
+        };
+        if (ck > 0) err = pair ? launch_rope(attn_tc5_kernel<true, true, false, true>, ck) : launch_rope(attn_tc5_kernel<false, true, false, true>, ck);
+        else err = pair ? launch_rope(attn_tc5_kernel<true, false, false, true>, 0) : launch_rope(attn_tc5_kernel<false, false, false, true>, 0);
+        if (err != cudaSuccess) return err;
+        ++*n_launches;
+        if (ck > 0 || own_merge) return cudaSuccess;
+        err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p)
+                   : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 8), dim3(128), 0, st, 0, p);
+        if (err != cudaSuccess) return err;
+        ++*n_launches;
+        return cudaSuccess;
+    }
     if (ck > 0) {
         // cluster form: the CTAs of a unit merge their partials through distributed shared memory; one launch
         err = paged ? (pair ? launch_attn(attn_tc5_kernel<true, true, true>, ck) : launch_attn(attn_tc5_kernel<false, true, true>, ck))

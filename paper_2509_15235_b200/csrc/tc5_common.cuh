@@ -366,6 +366,15 @@ __device__ __noinline__ void merge_unit(const MergeArgs m, int T, int geff, int 
 // pool [num_blocks][Hkv][page_rows][D] (tensor map (d, slot, block * Hkv + head)) or, token_major,
 // [num_blocks][page_rows][Hkv][D] (tensor map (d, head, block * page_rows + slot));
 // block_table[b][i] = pool block of logical slots [i * page_rows, (i + 1) * page_rows)
+// Fourth kernel parameter of the instantiations with the fused rotary embedding (they serve contiguous caches, so it
+// takes the place of PagedArgs; a larger common parameter block costs the other instantiations registers).
+struct RopeArgs {
+    const double2* rope_k;     // [B][N][D/2] (cos, sin) of positions * theta^(-2j/D), fp64: the k rows' rotation
+    const float2* rope_q;      // the same angles in fp32: the q rows' rotation (q is only consumed, never written back)
+    const __nv_bfloat16* k_new; const __nv_bfloat16* v_new;   // [B][N][Hkv][D] rows of the tree, to be placed at slots S + i
+    __nv_bfloat16* k_cache; __nv_bfloat16* v_cache;            // [B][Hkv][S_max][D]
+    int* unit_counters;        // as in PagedArgs
+};
 struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N, token_major; int* status;
                    int* unit_counters; };   // even split: arrivals per unit (all zero between calls); nullptr: a merge kernel follows
 

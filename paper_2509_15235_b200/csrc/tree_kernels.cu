@@ -332,7 +332,7 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
                  const __nv_bfloat16* __restrict__ v_new, const int32_t* __restrict__ positions,
                  const int32_t* __restrict__ kv_len, __nv_bfloat16* __restrict__ k_cache,
                  __nv_bfloat16* __restrict__ v_cache, double log2_theta, int N, int Hq, int Hkv, int D, int S_max,
-                 int* status, const RowMap rmap) {
+                 int* status, const RowMap rmap, __nv_bfloat16* __restrict__ q_out, const double2* __restrict__ table) {
     __shared__ double cs[64], sn[64];
     // First wait for the kernel before this one (q / k_new / v_new may come from it, and so may kv_len), only then let
     // the next kernel in: an attention call that follows reads kv_len and committed cache rows before its own wait,
@@ -353,9 +353,9 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
     const uint4* src = nullptr;
     uint4* dst = nullptr;
     if (row < Hq) {
-        __nv_bfloat16* r = q + (((size_t)b * N + i) * Hq + row) * D;
-        src = reinterpret_cast<const uint4*>(r);
-        dst = reinterpret_cast<uint4*>(r);
+        const size_t o = (((size_t)b * N + i) * Hq + row) * D;
+        src = reinterpret_cast<const uint4*>(q + o);
+        dst = reinterpret_cast<uint4*>(q_out + o);      // q itself, or a separate rotated copy
     } else if (row < rows) {
         const bool is_k = row < Hq + Hkv;
         const int hk = row - Hq - (is_k ? 0 : Hkv);
@@ -370,9 +370,14 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
         hi = src[(c8 + half) / 8];
     }
     if ((int)threadIdx.x < half) {
-        const double ang = (double)positions[(size_t)b * N + i] * exp2(-2.0 * (double)threadIdx.x / (double)D * log2_theta);
         double s_, c_;
-        sincos(ang, &s_, &c_);
+        if (table) {                                      // the same values, formed once per cycle by rope_table_kernel
+            const double2 t = table[((size_t)b * N + i) * half + threadIdx.x];
+            c_ = t.x; s_ = t.y;
+        } else {
+            const double ang = (double)positions[(size_t)b * N + i] * exp2(-2.0 * (double)threadIdx.x / (double)D * log2_theta);
+            sincos(ang, &s_, &c_);
+        }
         cs[threadIdx.x] = c_;
         sn[threadIdx.x] = s_;
     }
@@ -381,6 +386,30 @@ rope_rows_kernel(__nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict_
     if (row < Hq + Hkv) rope_rotate8(lo, hi, cs + c8, sn + c8);
     dst[c8 / 8] = lo;
     dst[(c8 + half) / 8] = hi;
+}
+
+namespace {
+// One block per (node, sequence), one thread per frequency: the angle and its sine and cosine exactly as
+// rope_rows_kernel forms them, stored once as fp64 and once rounded to fp32.
+__global__ void rope_table_kernel(const int32_t* __restrict__ positions, double log2_theta, int N, int D,
+                                  double2* __restrict__ tab64, float2* __restrict__ tab32) {
+    const int i = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
+    if (j >= D / 2) return;
+    const double ang = (double)positions[(size_t)b * N + i] * exp2(-2.0 * (double)j / (double)D * log2_theta);
+    double s_, c_;
+    sincos(ang, &s_, &c_);
+    const size_t o = ((size_t)b * N + i) * (D / 2) + j;
+    tab64[o] = make_double2(c_, s_);
+    tab32[o] = make_float2((float)c_, (float)s_);
+}
+}  // namespace
+
+cudaError_t launch_rope_table(const int32_t* positions, int B, int N, int D, float theta, void* table, cudaStream_t st) {
+    if (B * N == 0) return cudaSuccess;
+    double2* t64 = (double2*)table;
+    float2* t32 = (float2*)(t64 + (size_t)B * N * (D / 2));
+    rope_table_kernel<<<dim3(N, B), D / 2, 0, st>>>(positions, log2((double)theta), N, D, t64, t32);
+    return cudaGetLastError();
 }
 
 namespace {
@@ -407,7 +436,8 @@ cudaError_t launch_check_positions(const int32_t* positions, const int32_t* kv_l
 cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, const int32_t* positions,
                              const int32_t* kv_len, void* k_cache, void* v_cache, float theta, int B, int N, int Hq,
                              int Hkv, int D, int S_max, int* status, cudaStream_t st, const int32_t* block_table,
-                             int table_stride, int page_rows, int num_blocks, int token_major) {
+                             int table_stride, int page_rows, int num_blocks, int token_major, void* q_out,
+                             const void* angle_table) {
     if (B == 0) return cudaSuccess;
     const RowMap rmap = {block_table, table_stride, page_rows, num_blocks, token_major};
     cudaLaunchConfig_t cfg = {};
@@ -422,7 +452,8 @@ cudaError_t launch_rope_rows(void* q, const void* k_new, const void* v_new, cons
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, rope_rows_kernel, (__nv_bfloat16*)q, (const __nv_bfloat16*)k_new,
                               (const __nv_bfloat16*)v_new, positions, kv_len, (__nv_bfloat16*)k_cache,
-                              (__nv_bfloat16*)v_cache, log2((double)theta), N, Hq, Hkv, D, S_max, status, rmap);
+                              (__nv_bfloat16*)v_cache, angle_table ? 0.0 : log2((double)theta), N, Hq, Hkv, D, S_max, status,
+                              rmap, (__nv_bfloat16*)(q_out ? q_out : q), (const double2*)angle_table);
 }
 
 // ------------------------------------------------------------------------------------------------

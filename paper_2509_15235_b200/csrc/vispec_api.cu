@@ -13,7 +13,12 @@ size_t workspace_bytes(const vispec_shape& s, int sm_count) {
     const size_t slot = slot_bytes(s.D);
     // generic kernel: at most 4*SMs + units partials of 64 rows (half slots);
     // persistent kernel: at most two partials of 128 rows per CTA, one CTA per SM.
-    return kCounterBytes + (4 * (size_t)sm_count + units64) * (slot / 2) + 2 * (size_t)sm_count * slot;
+    return kCounterBytes + (4 * (size_t)sm_count + units64) * (slot / 2) + 2 * (size_t)sm_count * slot + q_scratch_bytes(s);
+}
+
+// Rotated copy of q for the fused rotary call where it runs as two kernels: the last q_scratch_bytes of the workspace.
+size_t q_scratch_bytes(const vispec_shape& s) {
+    return ((size_t)s.B_max * s.N_max * s.Hq * s.D * 2 + 255) / 256 * 256;
 }
 
 }  // namespace vispec
@@ -122,7 +127,8 @@ int vispec_ctx_set_workspace(vispec_ctx* c, void* ws, size_t bytes) {
     if (cudaMemset(ws, 0, kCounterBytes) != cudaSuccess) return VISPEC_E_CUDA;
     if (cudaDeviceSynchronize() != cudaSuccess) return VISPEC_E_CUDA;
     c->ws = ws;
-    c->ws_bytes = bytes;
+    c->ws_bytes_used = workspace_bytes(c->shape, c->sm_count);
+    c->ws_bytes = bytes - q_scratch_bytes(c->shape);    // what the attention kernels may use for partials
     return VISPEC_OK;
 }
 
@@ -262,6 +268,66 @@ int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void*
         err = launch_check_positions(positions, kv_len, tree_mask, B, N, c->d_status, (cudaStream_t)stream);
         c->launches += 1;
     }
+    return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
+}
+
+int vispec_rope_table_bytes(const vispec_ctx* c, int B, int N, size_t* out) {
+    if (!c || !out) return VISPEC_E_NULL;
+    if (B < 0 || N < 0) return VISPEC_E_SHAPE;
+    *out = (size_t)B * N * (c->shape.D / 2) * (sizeof(double) * 2 + sizeof(float) * 2);
+    return VISPEC_OK;
+}
+
+int vispec_rope_table_build(vispec_ctx* c, const int32_t* positions, int B, int N, float theta, void* table,
+                            void* stream) {
+    if (!c || !positions || !table) return VISPEC_E_NULL;
+    if (!aligned(table, 16)) return VISPEC_E_ALIGN;
+    if (B < 0 || B > c->shape.B_max || N < 1 || N > c->shape.N_max || !(theta > 1.f)) return VISPEC_E_SHAPE;
+    if (launch_rope_table(positions, B, N, c->shape.D, theta, table, (cudaStream_t)stream) != cudaSuccess) return VISPEC_E_CUDA;
+    if (B > 0) c->launches += 1;
+    return VISPEC_OK;
+}
+
+int vispec_tree_verify_attn_rope(vispec_ctx* c, int layer, const void* q, const void* k_new, const void* v_new,
+                                 const void* rope_table, const int32_t* kv_len, const uint64_t* tree_mask, int B, int N,
+                                 float scale, void* out, float* lse, void* stream) {
+    if (!c || !q || !k_new || !v_new || !rope_table || !kv_len || !tree_mask || !out) return VISPEC_E_NULL;
+    if (!aligned(q, 16) || !aligned(out, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(rope_table, 16))
+        return VISPEC_E_ALIGN;
+    const vispec_shape& s = c->shape;
+    if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
+    if (layer < 0 || layer >= s.layers) return VISPEC_E_RANGE;
+    if (!c->h_k[layer]) return VISPEC_E_UNREGISTERED;
+    if (c->page_rows[layer]) return VISPEC_E_UNSUPPORTED;
+    if (!c->ws) return VISPEC_E_WORKSPACE;
+    if (B == 0) return VISPEC_OK;
+    AttnArgs a = {};
+    a.q = q; a.k = c->h_k[layer]; a.v = c->h_v[layer];
+    a.kv_len = kv_len; a.mask = tree_mask; a.out = out; a.lse = lse;
+    a.B = B; a.N = N; a.Hq = s.Hq; a.Hkv = s.Hkv; a.D = s.D; a.S_max = s.S_max;
+    a.scale = scale; a.ws = c->ws; a.ws_bytes = c->ws_bytes; a.status = c->d_status;
+    a.sm_count = c->sm_count;
+    a.early_prefetch = c->early_prefetch;
+    a.tc5_path = c->tc5_path;
+    a.kv_len_hint = c->kv_len_hint;
+    a.k_map = &c->k_map[layer]; a.v_map = &c->v_map[layer];
+    a.rope_table = rope_table; a.k_new = k_new; a.v_new = v_new;
+    if (c->force_generic || !attn_tc5_supports(a)) return VISPEC_E_UNSUPPORTED;
+    int n = 0;
+    cudaError_t err = cudaSuccess;
+    if (!attn_tc5_uses_clusters(a)) {
+        // Where the kernel splits its work evenly over the SMs (many units, long caches) the in-kernel rotation costs
+        // more than it saves: the rows go through the rotation kernel instead (the table in place of positions, q into
+        // the scratch copy at the end of the workspace so that the caller's q stays as it is), then the plain attention.
+        void* q_rot = (unsigned char*)c->ws + c->ws_bytes_used - q_scratch_bytes(s);
+        err = launch_rope_rows(const_cast<void*>(q), k_new, v_new, nullptr, kv_len, c->h_k[layer], c->h_v[layer], 0.f, B, N,
+                               s.Hq, s.Hkv, s.D, s.S_max, c->d_status, (cudaStream_t)stream, nullptr, 0, 0, 0, 0, q_rot,
+                               rope_table);
+        c->launches += 1;
+        a.q = q_rot; a.rope_table = nullptr; a.k_new = nullptr; a.v_new = nullptr;
+    }
+    if (err == cudaSuccess) err = launch_attn_tc5(a, (cudaStream_t)stream, &n);
+    c->launches += n;
     return err == cudaSuccess ? VISPEC_OK : VISPEC_E_CUDA;
 }
 

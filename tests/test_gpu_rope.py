@@ -156,3 +156,67 @@ def test_commit_then_rope_then_attention_chained_on_one_stream(Hq, Hkv):
         assert np.abs(out.float().cpu().numpy() - want).max() <= 2e-2
         assert np.abs(lse.cpu().numpy() - want_lse).max() <= 2e-3
         ctx.close()
+
+
+@pytest.mark.parametrize("split_form", [0, 1, 2, 3])
+@pytest.mark.parametrize("B,N,Hq,Hkv,kv_len,S_max", [
+    (1, 60, 8, 8, [1100], 1280),            # one row block per head, several tiles, tree rows inside one tile
+    (2, 60, 4, 4, [1000, 350], 1152),       # tree rows straddle a tile boundary (1000 + 60 > 1024); two sequences
+    (2, 60, 14, 2, [533, 472], 640),        # 7 query heads per kv head: four row blocks share the tree rows
+    (1, 31, 8, 2, [97], 256),               # the paper's tree; the first tile already holds tree rows
+])
+def test_fused_rope_attention_matches_rope_then_attention_of_the_oracle(B, N, Hq, Hkv, kv_len, S_max, split_form):
+    """vispec_tree_verify_attn_rope against oracle.rope_rows followed by oracle.tree_attn: the cache afterwards (v rows and
+    untouched slots bit-exact, rotated k rows within one bf16 step on at most 1e-4 of the elements), q untouched, and
+    the attention output within its tolerance."""
+    from paper_2509_15235_b200 import binding
+    import gpu_util as gu
+    D = 128
+    rng = np.random.Generator(np.random.Philox(900 + N + Hq))
+    kv_len = np.asarray(kv_len, dtype=np.int32)
+    q = synth.normal_bf16((B, N, Hq, D), 801); k = synth.normal_bf16((B, N, Hkv, D), 802)
+    v = synth.normal_bf16((B, N, Hkv, D), 803)
+    kc = synth.normal_bf16((B, Hkv, S_max, D), 804); vc = synth.normal_bf16((B, Hkv, S_max, D), 805)
+    parents = np.stack([synth.draw_tree(N, 6, 4, rng) for _ in range(B)])
+    mask, depth, _ = oracle.tree_mask(parents)
+    positions = (kv_len[:, None] + depth).astype(np.int32)
+    theta, scale = 1e6, 1.0 / np.sqrt(D)
+    o_q, o_k, o_v, skipped = oracle.rope_rows(q, k, v, positions, kv_len, kc, vc, theta)
+    assert skipped == 0
+    want, want_lse = oracle.tree_attn(o_q, o_k, o_v, kv_len, mask, scale)
+
+    ctx = binding.VerifyContext(B, N, Hq, Hkv, D, S_max, 1)
+    if split_form:
+        ctx.ctx_set_option(binding.OPT_SPLIT_FORM, split_form)
+    kd, vd, qd = gu.bf16_dev(kc), gu.bf16_dev(vc), gu.bf16_dev(q)
+    ctx.cache_register(0, kd, vd)
+    table = ctx.rope_table_build(gu.i32_dev(positions), theta)
+    out = torch.full((B, N, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, Hq, N), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.tree_verify_attn_rope(0, qd, gu.bf16_dev(k), gu.bf16_dev(v), table, gu.i32_dev(kv_len), gu.u64_dev(mask), scale, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.status_poll() == 0
+    assert np.array_equal(gu.bf16_bits(qd), q)                      # q is read only
+    assert np.array_equal(gu.bf16_bits(vd), o_v)                    # copies and untouched slots: exact
+    step = np.abs(_ordered(gu.bf16_bits(kd)) - _ordered(o_k))
+    assert step.max() <= 1 and (step != 0).mean() <= 1e-4
+    assert np.abs(out.float().cpu().numpy() - want).max() <= 2e-2
+    assert np.abs(lse.cpu().numpy() - want_lse).max() <= 2e-3
+    ctx.close()
+
+
+def test_fused_rope_attention_refuses_what_it_does_not_serve():
+    from paper_2509_15235_b200 import binding
+    ctx = binding.VerifyContext(1, 8, 2, 2, 64, 128, 1)            # head size 64: the generic kernel's territory
+    c = torch.zeros((1, 2, 128, 64), dtype=torch.bfloat16, device="cuda")
+    ctx.cache_register(0, c, c.clone())
+    q = torch.zeros((1, 8, 2, 64), dtype=torch.bfloat16, device="cuda")
+    pos = torch.zeros((1, 8), dtype=torch.int32, device="cuda")
+    table = ctx.rope_table_build(pos, 1e4)
+    with pytest.raises(binding.VispecError) as e:
+        ctx.tree_verify_attn_rope(0, q, q.clone(), q.clone(), table, pos[:, 0].contiguous(),
+                                  torch.ones((1, 8, 1), dtype=torch.int64, device="cuda"), 0.1, q.clone())
+    assert e.value.code == -5
+    with pytest.raises(binding.VispecError):
+        ctx.rope_table_build(pos, 1.0)
+    ctx.close()
