@@ -209,6 +209,45 @@ __device__ __forceinline__ void rope8_f32(uint4& lo, uint4& hi, const float2* cs
         b[t] = __float2bfloat16_rn(y * cs[t].x + x * cs[t].y);
     }
 }
+// The Q tile of a segment, rotated on the way in: softmax thread st takes the chunk pair (c, c + 8) of rows st/8,
+// st/8 + 32, ... with its eight (cos, sin) pairs; every load is issued before the first use.  Not inlined, like the row
+// placement below: what the kernel's hot loops share the instruction cache with is kept small.
+template <bool PAIR, int ROWS>
+__device__ __noinline__ void load_q_rotated(unsigned char* sm, const __nv_bfloat16* __restrict__ q, const float2* __restrict__ rope_q,
+                                            int b, int kvh, int mblock, int rows_total, int G, int N, int Hq, int st) {
+    constexpr int PITEMS = ROWS * 8 / kSmx;
+    const int c = st & 7;
+    uint4 lo[PITEMS], hi[PITEMS];
+    float4 tab[PITEMS][4];
+#pragma unroll
+    for (int k = 0; k < PITEMS; ++k) {
+        const int row = mblock * 128 + (st >> 3) + 32 * k;
+        lo[k] = make_uint4(0, 0, 0, 0); hi[k] = lo[k];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) tab[k][j] = make_float4(1.f, 0.f, 1.f, 0.f);
+        if (row < rows_total) {
+            const int node = row / G, head = kvh * G + row % G;
+            const uint4* src = reinterpret_cast<const uint4*>(q + (((size_t)b * N + node) * Hq + head) * D);
+            lo[k] = src[c]; hi[k] = src[c + 8];
+            const float4* t4 = reinterpret_cast<const float4*>(rope_q + ((size_t)b * N + node) * (D / 2) + 8 * c);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) tab[k][j] = t4[j];
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < PITEMS; ++k) {
+        const int r = (st >> 3) + 32 * k;
+        rope8_f32(lo[k], hi[k], reinterpret_cast<const float2*>(tab[k]));
+        unsigned char* dst = sm + SMEM_Q + r * 128 + ((c ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(dst) = lo[k];
+        *reinterpret_cast<uint4*>(dst + HALF_BYTES) = hi[k];
+        if (PAIR) {
+            *reinterpret_cast<uint4*>(dst + 64 * 128) = lo[k];
+            *reinterpret_cast<uint4*>(dst + HALF_BYTES + 64 * 128) = hi[k];
+        }
+    }
+}
+
 // The tree rows of (sequence b, kv head kvh) with tree index in [t_lo, t_hi): k rotated, v copied, written to slots
 // S + t of the cache.  Run by the kSmx softmax threads (thread st) of the CTA whose steps contain those slots, right
 // after the Q tile; every load of a pass is issued before the first use.  Not inlined: its registers stay out of the
@@ -490,39 +529,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 if (!mbar_wait_warp(bar(B_XFREE), (seg - 1) & 1, abort_flag)) return false;
             }
             if constexpr (ROPE) {
-                // rotated on the way in: a thread takes the chunk pair (c, c + 8) of rows st/8, st/8 + 32, ... with its
-                // eight angles; all loads are issued before the first use
-                constexpr int PITEMS = ROWS * 8 / kSmx;
-                const int c = st & 7;
-                uint4 lo[PITEMS], hi[PITEMS];
-                float4 tab[PITEMS][4];
-#pragma unroll
-                for (int k = 0; k < PITEMS; ++k) {
-                    const int row = sg.mblock * 128 + (st >> 3) + 32 * k;
-                    lo[k] = make_uint4(0, 0, 0, 0); hi[k] = lo[k];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) tab[k][j] = make_float4(1.f, 0.f, 1.f, 0.f);
-                    if (row < rows_total) {
-                        const int node = row / G, head = sg.kvh * G + row % G;
-                        const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)sg.b * N + node) * p.Hq + head) * D);
-                        lo[k] = src[c]; hi[k] = src[c + 8];
-                        const float4* t4 = reinterpret_cast<const float4*>(pa.rope_q + ((size_t)sg.b * N + node) * (D / 2) + 8 * c);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) tab[k][j] = t4[j];
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < PITEMS; ++k) {
-                    const int r = (st >> 3) + 32 * k;
-                    rope8_f32(lo[k], hi[k], reinterpret_cast<const float2*>(tab[k]));
-                    unsigned char* dst = sm + SMEM_Q + r * 128 + ((c ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4*>(dst) = lo[k];
-                    *reinterpret_cast<uint4*>(dst + HALF_BYTES) = hi[k];
-                    if (PAIR) {
-                        *reinterpret_cast<uint4*>(dst + 64 * 128) = lo[k];
-                        *reinterpret_cast<uint4*>(dst + HALF_BYTES + 64 * 128) = hi[k];
-                    }
-                }
+                load_q_rotated<PAIR, ROWS>(sm, p.q, pa.rope_q, sg.b, sg.kvh, sg.mblock, rows_total, G, N, p.Hq, st);
                 fence_async_smem();
                 mbar_arrive(bar(B_QFULL));
                 return true;
