@@ -3,6 +3,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "vispec_internal.h"
 
 namespace vispec {
@@ -26,6 +28,13 @@ size_t q_scratch_bytes(const vispec_shape& s) {
 using namespace vispec;
 
 namespace {
+
+// One NVTX range per hot entry point (a no-op costing a few nanoseconds unless a profiler is attached).
+struct ApiRange {
+    explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+    ~ApiRange() { nvtxRangePop(); }
+};
+#define VISPEC_RANGE() ApiRange api_range_(__func__)
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -229,6 +238,7 @@ int vispec_cache_register_paged(vispec_ctx* c, int layer, void* k_pool, void* v_
 
 int vispec_tree_mask_build(vispec_ctx* c, const int32_t* parents, int B, int N, uint64_t* tree_mask,
                            int32_t* depth, void* stream) {
+    VISPEC_RANGE();
     if (!c || !parents || !tree_mask) return VISPEC_E_NULL;
     if (B < 0 || B > c->shape.B_max || N < 1 || N > c->shape.N_max) return VISPEC_E_SHAPE;
     if (launch_tree_mask(parents, B, N, tree_mask, depth, c->d_status, (cudaStream_t)stream) != cudaSuccess)
@@ -240,6 +250,7 @@ int vispec_tree_mask_build(vispec_ctx* c, const int32_t* parents, int B, int N, 
 int vispec_tree_verify_attn(vispec_ctx* c, int layer, const void* q, const void* k_cache, const void* v_cache,
                             const int32_t* kv_len, const uint64_t* tree_mask, const int32_t* positions,
                             int B, int N, float scale, void* out, float* lse, void* stream) {
+    VISPEC_RANGE();
     if (!c || !q || !kv_len || !tree_mask || !out) return VISPEC_E_NULL;
     if (!aligned(q, 16) || !aligned(out, 16)) return VISPEC_E_ALIGN;
     const vispec_shape& s = c->shape;
@@ -280,6 +291,7 @@ int vispec_rope_table_bytes(const vispec_ctx* c, int B, int N, size_t* out) {
 
 int vispec_rope_table_build(vispec_ctx* c, const int32_t* positions, int B, int N, float theta, void* table,
                             void* stream) {
+    VISPEC_RANGE();
     if (!c || !positions || !table) return VISPEC_E_NULL;
     if (!aligned(table, 16)) return VISPEC_E_ALIGN;
     if (B < 0 || B > c->shape.B_max || N < 1 || N > c->shape.N_max || !(theta > 1.f)) return VISPEC_E_SHAPE;
@@ -291,6 +303,7 @@ int vispec_rope_table_build(vispec_ctx* c, const int32_t* positions, int B, int 
 int vispec_tree_verify_attn_rope(vispec_ctx* c, int layer, const void* q, const void* k_new, const void* v_new,
                                  const void* rope_table, const int32_t* kv_len, const uint64_t* tree_mask, int B, int N,
                                  float scale, void* out, float* lse, void* stream) {
+    VISPEC_RANGE();
     if (!c || !q || !k_new || !v_new || !rope_table || !kv_len || !tree_mask || !out) return VISPEC_E_NULL;
     if (!aligned(q, 16) || !aligned(out, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(rope_table, 16))
         return VISPEC_E_ALIGN;
@@ -334,6 +347,7 @@ int vispec_tree_verify_attn_rope(vispec_ctx* c, int layer, const void* q, const 
 int vispec_tree_verify_attn_paged(vispec_ctx* c, int layer, const void* q, const int32_t* kv_len,
                                   const int32_t* block_table, int table_stride, const uint64_t* tree_mask, int B, int N,
                                   float scale, void* out, float* lse, void* stream) {
+    VISPEC_RANGE();
     if (!c || !q || !kv_len || !block_table || !tree_mask || !out) return VISPEC_E_NULL;
     if (!aligned(q, 16) || !aligned(out, 16)) return VISPEC_E_ALIGN;
     const vispec_shape& s = c->shape;
@@ -367,6 +381,7 @@ int vispec_tree_verify_attn_paged(vispec_ctx* c, int layer, const void* q, const
 int vispec_kv_compact_paged(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* path,
                             const int32_t* accept_len, const int32_t* kv_len, const int32_t* block_table,
                             int table_stride, int32_t* kv_len_out, int B, int N, void* stream) {
+    VISPEC_RANGE();
     if (!c || !path || !accept_len || !kv_len || !block_table) return VISPEC_E_NULL;
     const vispec_shape& s = c->shape;
     if (B < 0 || B > s.B_max || N < 1 || N > s.N_max || table_stride < 1) return VISPEC_E_SHAPE;
@@ -407,6 +422,7 @@ int vispec_accept_commit_paged(vispec_ctx* c, int layer_begin, int layer_end, co
                                const int32_t* target_ids, const int32_t* parents, const int32_t* kv_len,
                                const int32_t* block_table, int table_stride, int B, int N, int32_t* path,
                                int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, void* stream) {
+    VISPEC_RANGE();
     if (!c || !draft_ids || !target_ids || !parents || !kv_len || !block_table || !path || !accept_len || !bonus)
         return VISPEC_E_NULL;
     const vispec_shape& s = c->shape;
@@ -428,6 +444,7 @@ int vispec_accept_commit_paged(vispec_ctx* c, int layer_begin, int layer_end, co
 int vispec_rope_tree_rows_paged(vispec_ctx* c, int layer, void* q, const void* k_new, const void* v_new,
                                 const int32_t* positions, const int32_t* kv_len, const int32_t* block_table,
                                 int table_stride, int B, int N, float theta, void* stream) {
+    VISPEC_RANGE();
     if (!c || !q || !k_new || !v_new || !positions || !kv_len || !block_table) return VISPEC_E_NULL;
     if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return VISPEC_E_ALIGN;
     const vispec_shape& s = c->shape;
@@ -446,6 +463,7 @@ int vispec_rope_tree_rows_paged(vispec_ctx* c, int layer, void* q, const void* k
 
 int vispec_rope_tree_rows(vispec_ctx* c, int layer, void* q, const void* k_new, const void* v_new,
                           const int32_t* positions, const int32_t* kv_len, int B, int N, float theta, void* stream) {
+    VISPEC_RANGE();
     if (!c || !q || !k_new || !v_new || !positions || !kv_len) return VISPEC_E_NULL;
     if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return VISPEC_E_ALIGN;
     const vispec_shape& s = c->shape;
@@ -461,6 +479,7 @@ int vispec_rope_tree_rows(vispec_ctx* c, int layer, void* q, const void* k_new, 
 }
 
 int vispec_stream_probe(vispec_ctx* c, int layer, const int32_t* kv_len, int B, int N, void* stream) {
+    VISPEC_RANGE();
     if (!c || !kv_len) return VISPEC_E_NULL;
     const vispec_shape& s = c->shape;
     if (B < 1 || B > s.B_max || B > 32 || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
@@ -480,6 +499,7 @@ int vispec_stream_probe(vispec_ctx* c, int layer, const int32_t* kv_len, int B, 
 
 int vispec_accept(vispec_ctx* c, const int32_t* draft_ids, const int32_t* target_ids, const int32_t* parents,
                   int B, int N, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
+    VISPEC_RANGE();
     if (!c || !draft_ids || !target_ids || !parents || !path || !accept_len || !bonus) return VISPEC_E_NULL;
     if (B < 0 || B > c->shape.B_max || N < 1 || N > c->shape.N_max) return VISPEC_E_SHAPE;
     if (launch_accept(draft_ids, target_ids, parents, B, N, path, accept_len, bonus, c->d_status,
@@ -491,6 +511,7 @@ int vispec_accept(vispec_ctx* c, const int32_t* draft_ids, const int32_t* target
 
 int vispec_tree_rerank(vispec_ctx* c, const int32_t* cand_parent, const int32_t* cand_token, const float* cand_score,
                        int B, int M, int K, int32_t* parents, int32_t* draft_ids, int32_t* selected, void* stream) {
+    VISPEC_RANGE();
     if (!c || !cand_parent || !cand_token || !cand_score || !parents || !draft_ids || (!selected && K > 0))
         return VISPEC_E_NULL;
     if (B < 0 || B > c->shape.B_max || M < 1 || M > 2048 || K < 0 || K > M || K + 1 > c->shape.N_max)
@@ -505,6 +526,7 @@ int vispec_tree_rerank(vispec_ctx* c, const int32_t* cand_parent, const int32_t*
 int vispec_accept_sampled(vispec_ctx* c, const int32_t* draft_ids, const int32_t* parents, const float* p_target,
                           const float* p_draft, const float* u_accept, const float* u_bonus, int B, int N, int V,
                           int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
+    VISPEC_RANGE();
     if (!c || !draft_ids || !parents || !p_target || !p_draft || !u_accept || !u_bonus || !path || !accept_len || !bonus)
         return VISPEC_E_NULL;
     if (!aligned(p_target, 16) || !aligned(p_draft, 16)) return VISPEC_E_ALIGN;
@@ -519,6 +541,7 @@ int vispec_accept_sampled(vispec_ctx* c, const int32_t* draft_ids, const int32_t
 int vispec_kv_compact(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* path,
                       const int32_t* accept_len, const int32_t* kv_len, int32_t* kv_len_out, int B, int N,
                       void* stream) {
+    VISPEC_RANGE();
     if (!c || !path || !accept_len || !kv_len) return VISPEC_E_NULL;
     const vispec_shape& s = c->shape;
     if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;
@@ -538,6 +561,7 @@ int vispec_kv_compact(vispec_ctx* c, int layer_begin, int layer_end, const int32
 int vispec_accept_commit(vispec_ctx* c, int layer_begin, int layer_end, const int32_t* draft_ids,
                          const int32_t* target_ids, const int32_t* parents, const int32_t* kv_len, int B, int N,
                          int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* kv_len_out, void* stream) {
+    VISPEC_RANGE();
     if (!c || !draft_ids || !target_ids || !parents || !kv_len || !path || !accept_len || !bonus) return VISPEC_E_NULL;
     const vispec_shape& s = c->shape;
     if (B < 0 || B > s.B_max || N < 1 || N > s.N_max) return VISPEC_E_SHAPE;

@@ -71,3 +71,25 @@ def test_reference_arm_runs_on_rank_zero_only():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
     assert outs[1].strip() == ""                             # the other rank exits 0 without work
+
+
+def test_the_roofline_names_the_binding_bound_of_each_workload():
+    """bench.attention_roofline on the workload shapes: multi-head 60-node trees are bound by HBM, the grouped-query
+    ones (7 or 8 query heads per kv head, 60 nodes) by the tensor cores, and the fraction is the floor over the time."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2509_15235_b200 import synth
+    hbm, tflops, mhz, _ = bench.measured_peaks()
+    for name, want in (("llava7b", "hbm"), ("llava13b_b4", "hbm"), ("qwen3b_S8192_N16_B4", "hbm"),
+                       ("qwen7b", "tensor"), ("qwen3b_S8192_N60_B4", "tensor"), ("qwen3b_S32768_N128_B8", "tensor")):
+        cfg = synth.get_config(name)
+        kv_len = synth.make_tree_inputs(cfg)["kv_len"]
+        r = bench.attention_roofline(cfg, kv_len, 20.0, 148)
+        assert r["bound"] == want, (name, r)
+        assert abs(r["frac"] - r["floor_us"][want] / 20.0) < 1e-9
+        assert r["floor_us"][want] == max(r["floor_us"].values())
+        kv_bytes = cfg.kv_bytes_per_layer(kv_len)
+        assert abs(r["kv_gbs"] - kv_bytes / 20e-6 / 1e9) < 1e-6
+        assert abs(r["floor_us"]["hbm"] - kv_bytes / (hbm * 1e9) * 1e6) < 1e-9
+        tokens = sum(int(s) + cfg.N for s in kv_len) * cfg.Hkv
+        assert abs(r["floor_us"]["tensor"] - tokens * 4 * cfg.D * cfg.G * cfg.N / (tflops * 1e12) * 1e6) < 1e-9
