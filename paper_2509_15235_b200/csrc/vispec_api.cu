@@ -137,7 +137,7 @@ int vispec_ctx_set_workspace(vispec_ctx* c, void* ws, size_t bytes) {
     if (cudaDeviceSynchronize() != cudaSuccess) return VISPEC_E_CUDA;
     c->ws = ws;
     c->ws_bytes_used = workspace_bytes(c->shape, c->sm_count);
-    c->ws_bytes = bytes - q_scratch_bytes(c->shape);    // what the attention kernels may use for partials
+    c->ws_bytes = c->ws_bytes_used - q_scratch_bytes(c->shape);   // what the attention kernels may use for partials
     return VISPEC_OK;
 }
 
