@@ -24,7 +24,8 @@
 //   warp 1     issuer (one thread) of S = Q K^T as 128x128x16 tcgen05.mma; owns the TMEM allocation
 //   warp 2     issuer (one thread) of O += P V; the two chains wait on different barriers, so each has its own
 //              thread and neither's waits delay the other's instructions
-//   warp 3     derives the schedule from kv_len, then idles
+//   warp 3     derives the schedule from kv_len; with at most 64 rows per unit and a contiguous cache its lane 0
+//              then produces the V ring, so that warp 0's K copies never queue behind a wait for a V stage
 //   warps 4-11 softmax: thread <-> TMEM lane; warps w and w+4 share the same 32 accumulator rows and each takes
 //              half of a step's columns (the row maximum is exchanged through shared memory), so a row costs
 //              no shuffles; they also load Q at the start of every segment and run the segment epilogue
@@ -304,6 +305,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     static_assert(!(ROPE && PAGED), "the fused rotary embedding serves contiguous caches");
     constexpr int ROWS = PAIR ? 64 : 128;      // distinct query rows per CTA
     constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
+    constexpr bool SPLIT_V = PAIR && !PAGED;   // the V ring has a producer thread of its own (the spare warp's lane 0)
     extern __shared__ __align__(1024) unsigned char sm[];
     // the schedule hangs on kv_len, and a CTA that starts after its predecessor kernel has ended hangs on the
     // schedule: the load goes out first
@@ -412,17 +414,20 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                         if (!seg_counted) { ++nseg; seg_counted = true; }      // this segment has tree rows
                         if (!rows_placed(rows_done, nseg * kSmx, abort_flag)) { ok = false; break; }
                     }
-                    const int sk = it % NSK, sv = it % NSV;
+                    const int sk = it % NSK;
                     if (!mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(bar(B_KFULL + sk), STAGE_BYTES);
                     tma_load_3d(base + SMEM_K + sk * STAGE_BYTES, &k_map, bar(B_KFULL + sk), 0, tok, bh, pol);
                     tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES, &k_map, bar(B_KFULL + sk), 64, tok, bh, pol);
                     ++nk;
-                    if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(bar(B_VFULL + sv), STAGE_BYTES);
-                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES, &v_map, bar(B_VFULL + sv), 0, tok, bh, pol);
-                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES, &v_map, bar(B_VFULL + sv), 64, tok, bh, pol);
-                    ++nv;
+                    if constexpr (!SPLIT_V) {
+                        const int sv = it % NSV;
+                        if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(bar(B_VFULL + sv), STAGE_BYTES);
+                        tma_load_3d(base + SMEM_V + sv * STAGE_BYTES, &v_map, bar(B_VFULL + sv), 0, tok, bh, pol);
+                        tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES, &v_map, bar(B_VFULL + sv), 64, tok, bh, pol);
+                        ++nv;
+                    }
                 }
             }
             if (*abort_flag && lane == 0) {
@@ -430,6 +435,44 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 volatile int never = 0;
                 for (int u = max(0, nk - NSK); u < nk; ++u) mbar_wait(bar(B_KFULL + u % NSK), (u / NSK) & 1, &never);
                 for (int u = max(0, nv - NSV); u < nv; ++u) mbar_wait(bar(B_VFULL + u % NSV), (u / NSV) & 1, &never);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 3) {
+        // ================= TMA producer of the V ring (contiguous caches, rows <= 64) =================
+        // A V stage is free only after the PV product of the step it held, a softmax later than the K stage of the
+        // same step: one thread issuing both in order holds the K copies back behind every wait for a V stage.
+        // Measured in one call, one thread against two: 17.70 -> 17.50 us per layer on llava7b, 17.11 -> 16.91 on
+        // paper_tree, 71.4 -> 71.0 on llava13b_b4; with 128 rows per unit the two threads lose 1 % (16.43 -> 16.59 on
+        // qwen7b, 63.3 -> 63.8 on qwen3b_S32768_N16_B8), so those keep the single producer.
+        if (SPLIT_V && lane == 0 && active) {
+            const uint64_t pol = l2_evict_first_policy();
+            bool waited = !p.early;
+            int it = 0;
+            bool ok = true;
+            SegIter si = make_iter();
+            Seg sg;
+            int nseg = 0;
+            while (ok && si.next(sg)) {
+                const int bh = sg.b * p.Hkv + sg.kvh;
+                bool seg_counted = false;
+                for (int t = 0; t < sg.n; ++t, ++it) {
+                    const int tok = (sg.st0 + t) * STEP;
+                    if (!waited && tok + STEP > sg.S) { pdl_wait(); waited = true; }
+                    if (ROPE && tok + STEP > sg.S) {
+                        if (!seg_counted) { ++nseg; seg_counted = true; }
+                        if (!rows_placed(rows_done, nseg * kSmx, abort_flag)) { ok = false; break; }
+                    }
+                    const int sv = it % NSV;
+                    if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(bar(B_VFULL + sv), STAGE_BYTES);
+                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES, &v_map, bar(B_VFULL + sv), 0, tok, bh, pol);
+                    tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES, &v_map, bar(B_VFULL + sv), 64, tok, bh, pol);
+                }
+            }
+            if (*abort_flag) {
+                volatile int never = 0;
+                for (int u = max(0, it - NSV); u < it; ++u) mbar_wait(bar(B_VFULL + u % NSV), (u / NSV) & 1, &never);
             }
         }
         __syncwarp();
