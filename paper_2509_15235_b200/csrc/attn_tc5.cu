@@ -84,7 +84,9 @@ constexpr uint32_t COL_S = 0, COL_O = 256, COL_P = 384;
 enum { B_KFULL = 0, B_KEMPTY = B_KFULL + NSK, B_VFULL = B_KEMPTY + NSK, B_VEMPTY = B_VFULL + NSV,
        B_SFULL = B_VEMPTY + NSV, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 2,
        B_QFULL = B_PVDONE + 2, B_PAIRX = B_QFULL + 1, B_XCH = B_PAIRX + 4, B_XFREE = B_XCH + 1,
-       B_SEGSYNC = B_XFREE + 1, B_COUNT = B_SEGSYNC + 1 };
+       B_SEGSYNC = B_XFREE + 1,
+       B_ROWS = B_SEGSYNC + 1,      // fused rotary embedding: every rank of the cluster has put its share of the tree rows into the cache
+       B_COUNT = B_ROWS + 1 };
 static_assert(B_COUNT * 8 + 20 <= BAR_BYTES, "barrier block too small");
 
 constexpr int SMEM_TABRING = SMEM_SCHED + ((int)sizeof(Sched) + 15) / 16 * 16;   // 8 steps x 8 block numbers (paged cache)
@@ -174,20 +176,6 @@ __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensor
 }
 
 // ---- fused rotary embedding ---------------------------------------------------------------------------
-// Bounded wait of the producer until `want` softmax threads have put their share of the tree rows into the cache
-// (each counts itself in shared memory once per segment that has tree rows).
-__device__ __forceinline__ bool rows_placed(volatile int* rows_done, int want, volatile int* abort_flag) {
-    long long t0 = 0;
-    for (uint32_t it = 0; *rows_done < want; ++it) {
-        if ((it & 63) == 63) {
-            if (*abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitCycles) { *abort_flag = 1; return false; }
-        }
-    }
-    return true;
-}
 // Eight pairs (x = element j of the lower half, y = element j + D/2) rotated by their angles: fp64 with one rounding
 // to bf16 for the k rows that go to the cache, fp32 for q rows (consumed by the product, never stored).
 __device__ __forceinline__ void rope8_f64(uint4& lo, uint4& hi, const double2* cs) {
@@ -210,12 +198,57 @@ __device__ __forceinline__ void rope8_f32(uint4& lo, uint4& hi, const float2* cs
         b[t] = __float2bfloat16_rn(y * cs[t].x + x * cs[t].y);
     }
 }
-// The Q tile of a segment, rotated on the way in: softmax thread st takes the chunk pair (c, c + 8) of rows st/8,
-// st/8 + 32, ... with its eight (cos, sin) pairs; every load is issued before the first use.  Not inlined, like the row
-// placement below: what the kernel's hot loops share the instruction cache with is kept small.
+// Prologue of a CTA with the fused rotary embedding (one function, so that both memory round trips overlap): the upper
+// half of the softmax threads fetches this rank's share of the tree rows, tree index in [t_lo, t_hi), of (sequence b,
+// kv head kvh): one item = (k row, pair of 16-byte chunks c and c + 8) with its eight fp64 (cos, sin) pairs, plus two
+// 16-byte chunks of v rows; then every thread fetches its part of the Q tile (chunk pair (c, c + 8) of rows st/8,
+// st/8 + 32, ... with eight fp32 pairs each); only then the k rows are rotated (fp64, one rounding: bit-compatible with the
+// rotation kernel) and written to slots S + t of the cache with the v rows, and the Q rows are rotated (fp32: they feed
+// the score product only) into the swizzled tile.  Shares of more than 16 rows take further passes after that.  Not
+// inlined: its registers stay out of the step loop's budget and its code out of the step loop's way.
 template <bool PAIR, int ROWS>
-__device__ __noinline__ void load_q_rotated(unsigned char* sm, const __nv_bfloat16* __restrict__ q, const float2* __restrict__ rope_q,
-                                            int b, int kvh, int mblock, int rows_total, int G, int N, int Hq, int st) {
+__device__ __noinline__ void rope_prologue(unsigned char* sm, const __nv_bfloat16* __restrict__ q, const RopeArgs p, int N_, int Hq,
+                                           int Hkv_, int S_max_, int G, int rows_total, int b, int kvh, int mblock, int S,
+                                           int t_lo, int t_hi, int st) {
+    constexpr int HALF = kSmx / 2;
+    const int ps = st - HALF;                     // >= 0: this thread places rows
+    const size_t cache_row0 = ((size_t)b * Hkv_ + kvh) * S_max_ + S;
+    const int nk = (t_hi - t_lo) * 8, nv = (t_hi - t_lo) * 16;
+    auto k_src = [&](int i) { return reinterpret_cast<const uint4*>(p.k_new + (((size_t)b * N_ + t_lo + (i >> 3)) * Hkv_ + kvh) * D); };
+    auto k_tab = [&](int i) { return p.rope_k + ((size_t)b * N_ + t_lo + (i >> 3)) * (D / 2) + 8 * (i & 7); };
+    auto v_src = [&](int i) { return reinterpret_cast<const uint4*>(p.v_new + (((size_t)b * N_ + t_lo + (i >> 4)) * Hkv_ + kvh) * D) + (i & 15); };
+    auto k_store = [&](int i, uint4& lo, uint4& hi, const double2* cs) {
+        rope8_f64(lo, hi, cs);
+        uint4* dst = reinterpret_cast<uint4*>(p.k_cache + (cache_row0 + t_lo + (i >> 3)) * D);
+        dst[i & 7] = lo; dst[(i & 7) + 8] = hi;
+    };
+    auto v_store = [&](int i, const uint4& x) { reinterpret_cast<uint4*>(p.v_cache + (cache_row0 + t_lo + (i >> 4)) * D)[i & 15] = x; };
+
+    // ---- tree rows, first pass (16 rows): loads
+    uint4 klo = make_uint4(0, 0, 0, 0), khi = klo, vx[2];
+    double2 cs[8];
+    const bool has_k = ps >= 0 && ps < nk;
+    if (has_k) {
+        const uint4* src = k_src(ps);
+        klo = src[ps & 7]; khi = src[(ps & 7) + 8];
+        const double2* tab = k_tab(ps);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cs[j] = tab[j];
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+        if (ps >= 0 && ps + HALF * u < nv) vx[u] = *v_src(ps + HALF * u);
+    // (with 128 rows per unit the Q tile alone takes 96 registers per thread: there the rows are finished first; timed in
+    // one call on qwen7b: 16.3 against 17.6 us per layer of a step with both sets of loads in flight)
+    auto finish_rows = [&]() {
+        if (has_k) k_store(ps, klo, khi, cs);
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            if (ps >= 0 && ps + HALF * u < nv) v_store(ps + HALF * u, vx[u]);
+    };
+    if (!PAIR) finish_rows();
+
+    // ---- Q tile: loads
     constexpr int PITEMS = ROWS * 8 / kSmx;
     const int c = st & 7;
     uint4 lo[PITEMS], hi[PITEMS];
@@ -228,13 +261,18 @@ __device__ __noinline__ void load_q_rotated(unsigned char* sm, const __nv_bfloat
         for (int j = 0; j < 4; ++j) tab[k][j] = make_float4(1.f, 0.f, 1.f, 0.f);
         if (row < rows_total) {
             const int node = row / G, head = kvh * G + row % G;
-            const uint4* src = reinterpret_cast<const uint4*>(q + (((size_t)b * N + node) * Hq + head) * D);
+            const uint4* src = reinterpret_cast<const uint4*>(q + (((size_t)b * N_ + node) * Hq + head) * D);
             lo[k] = src[c]; hi[k] = src[c + 8];
-            const float4* t4 = reinterpret_cast<const float4*>(rope_q + ((size_t)b * N + node) * (D / 2) + 8 * c);
+            const float4* t4 = reinterpret_cast<const float4*>(p.rope_q + ((size_t)b * N_ + node) * (D / 2) + 8 * c);
 #pragma unroll
             for (int j = 0; j < 4; ++j) tab[k][j] = t4[j];
         }
     }
+
+    // ---- tree rows, first pass: rotate and store
+    if (PAIR) finish_rows();
+
+    // ---- Q tile: rotate into shared memory
 #pragma unroll
     for (int k = 0; k < PITEMS; ++k) {
         const int r = (st >> 3) + 32 * k;
@@ -247,51 +285,25 @@ __device__ __noinline__ void load_q_rotated(unsigned char* sm, const __nv_bfloat
             *reinterpret_cast<uint4*>(dst + HALF_BYTES + 64 * 128) = hi[k];
         }
     }
-}
 
-// The tree rows of (sequence b, kv head kvh) with tree index in [t_lo, t_hi): k rotated, v copied, written to slots
-// S + t of the cache.  Run by the kSmx softmax threads (thread st) of the CTA whose steps contain those slots, right
-// after the Q tile; every load of a pass is issued before the first use.  Not inlined: its registers stay out of the
-// step loop's budget.
-__device__ __noinline__ void place_tree_rows(const RopeArgs p, int N_, int Hkv_, int S_max_, int b, int kvh, int S, int t_lo,
-                                             int t_hi, int st) {
-    const size_t cache_row0 = ((size_t)b * Hkv_ + kvh) * S_max_ + S;
-    const int nk = (t_hi - t_lo) * 8;             // k: one item = (row, pair of 16-byte chunks c and c + 8)
-    const int nv = (t_hi - t_lo) * 16;            // v: 16 chunks per row, copied
-    for (int i0 = st, j0 = st; i0 < nk || j0 < nv; i0 += kSmx * 2, j0 += kSmx * 4) {
-        uint4 lo[2], hi[2], x[4];
-        double2 cs[2][8];
+    // ---- tree rows beyond the first 16 of the share
+    if (ps >= 0) {
+        for (int i = ps + HALF, j = ps + 2 * HALF; i < nk || j < nv; i += HALF, j += 2 * HALF) {
+            const bool more_k = i < nk;
+            if (more_k) {
+                const uint4* src = k_src(i);
+                klo = src[i & 7]; khi = src[(i & 7) + 8];
+                const double2* tb = k_tab(i);
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int i = i0 + kSmx * u;
-            if (i < nk) {
-                const int t = t_lo + (i >> 3), c = i & 7;
-                const uint4* src = reinterpret_cast<const uint4*>(p.k_new + (((size_t)b * N_ + t) * Hkv_ + kvh) * D);
-                lo[u] = src[c]; hi[u] = src[c + 8];
-                const double2* tab = p.rope_k + ((size_t)b * N_ + t) * (D / 2) + 8 * c;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) cs[u][j] = tab[j];
+                for (int jj = 0; jj < 8; ++jj) cs[jj] = tb[jj];
             }
-        }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int i = j0 + kSmx * u;
-            if (i < nv) x[u] = reinterpret_cast<const uint4*>(p.v_new + (((size_t)b * N_ + t_lo + (i >> 4)) * Hkv_ + kvh) * D)[i & 15];
-        }
+            for (int u = 0; u < 2; ++u)
+                if (j + HALF * u < nv) vx[u] = *v_src(j + HALF * u);
+            if (more_k) k_store(i, klo, khi, cs);
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int i = i0 + kSmx * u;
-            if (i < nk) {
-                const int t = t_lo + (i >> 3), c = i & 7;
-                rope8_f64(lo[u], hi[u], cs[u]);
-                uint4* dst = reinterpret_cast<uint4*>(p.k_cache + (cache_row0 + t) * D);
-                dst[c] = lo[u]; dst[c + 8] = hi[u];
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int i = j0 + kSmx * u;
-            if (i < nv) reinterpret_cast<uint4*>(p.v_cache + (cache_row0 + t_lo + (i >> 4)) * D)[i & 15] = x[u];
+            for (int u = 0; u < 2; ++u)
+                if (j + HALF * u < nv) v_store(j + HALF * u, vx[u]);
         }
     }
 }
@@ -303,6 +315,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const Tc5Params p,
                 const std::conditional_t<ROPE, RopeArgs, PagedArgs> pa) {
     static_assert(!(ROPE && PAGED), "the fused rotary embedding serves contiguous caches");
+    static_assert(!ROPE || CL, "the fused rotary embedding exists in the cluster form only (the even split goes through the rotation kernel)");
     constexpr int ROWS = PAIR ? 64 : 128;      // distinct query rows per CTA
     constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
     constexpr bool SPLIT_V = PAIR && !PAGED;   // the V ring has a producer thread of its own (the spare warp's lane 0)
@@ -321,7 +334,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + SMEM_BAR + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SMEM_BAR + B_COUNT * 8 + 8);
     volatile int* seg_flag = abort_flag + 1;               // this CTA delivered the last partial of the unit just finished
-    volatile int* rows_done = abort_flag + 2;              // fused rotary embedding: segments whose tree rows are in the cache
     Sched& sched = *reinterpret_cast<Sched*>(sm + SMEM_SCHED);
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
@@ -341,8 +353,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         mbar_init(bar(B_QFULL), kSmx);
         mbar_init(bar(B_XCH), 128); mbar_init(bar(B_XFREE), 128);
         mbar_init(bar(B_SEGSYNC), kSmx);
+        if (ROPE) mbar_init(bar(B_ROWS), cluster_size());
         *abort_flag = 0;
-        *rows_done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -358,6 +370,11 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // Fused rotary embedding: the ranks signal one another's barriers, which must exist by then.  Everybody arrives at
+    // the cluster barrier here (relaxed: fence.mbarrier_init has published the barriers); a warp waits, as a whole,
+    // where it first needs the guarantee.
+    bool cl_waited = !ROPE;
+    if (ROPE) cluster_arrive();
 
     // Schedule.  Cluster form: cluster <-> unit, the CTA of rank r takes the r-th of k equal parts of the
     // unit's steps (an empty part still takes part in the exchange).  Otherwise: equal ranges of the line of
@@ -374,9 +391,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         const int unit = cta / ck, b = unit / upb, uib = unit - b * upb;
         cl_seg.b = b; cl_seg.kvh = uib / p.n_mblocks; cl_seg.mblock = uib - cl_seg.kvh * p.n_mblocks;
         cl_seg.steps = sched.steps[b]; cl_seg.S = sched.len[b];
-        // (with the fused rotary embedding the last rank also places the tree rows: the short shares go to the end)
-        cl_seg.st0 = ROPE ? (cr * cl_seg.steps + ck - 1) / ck : (cr * cl_seg.steps) / ck;
-        cl_seg.n = (ROPE ? ((cr + 1) * cl_seg.steps + ck - 1) / ck : ((cr + 1) * cl_seg.steps) / ck) - cl_seg.st0;
+        cl_seg.st0 = (cr * cl_seg.steps) / ck;
+        cl_seg.n = ((cr + 1) * cl_seg.steps) / ck - cl_seg.st0;
         cl_seg.slot = -1;
     }
     auto make_iter = [&]() {
@@ -403,16 +419,15 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     waited = (r >> 30) & 1u;
                 }
             }
-            int nseg = 0;                        // segments with tree rows met so far
             while (!PAGED && ok && si.next(sg)) {
                 const int bh = sg.b * p.Hkv + sg.kvh;
-                bool seg_counted = false;
                 for (int t = 0; t < sg.n; ++t, ++it) {
                     const int tok = (sg.st0 + t) * STEP;
                     if (!waited && tok + STEP > sg.S) { pdl_wait(); waited = true; }   // the tree's rows come from the preceding kernel
                     if (ROPE && tok + STEP > sg.S) {
-                        if (!seg_counted) { ++nseg; seg_counted = true; }      // this segment has tree rows
-                        if (!rows_placed(rows_done, nseg * kSmx, abort_flag)) { ok = false; break; }
+                        // the tile holds tree rows: every rank's share must be in the cache, and ordered before this copy
+                        if (!mbar_wait_cluster(bar(B_ROWS), 0, abort_flag)) { ok = false; break; }
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
                     }
                     const int sk = it % NSK;
                     if (!mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag)) { ok = false; break; }
@@ -452,16 +467,14 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             bool ok = true;
             SegIter si = make_iter();
             Seg sg;
-            int nseg = 0;
             while (ok && si.next(sg)) {
                 const int bh = sg.b * p.Hkv + sg.kvh;
-                bool seg_counted = false;
                 for (int t = 0; t < sg.n; ++t, ++it) {
                     const int tok = (sg.st0 + t) * STEP;
                     if (!waited && tok + STEP > sg.S) { pdl_wait(); waited = true; }
                     if (ROPE && tok + STEP > sg.S) {
-                        if (!seg_counted) { ++nseg; seg_counted = true; }
-                        if (!rows_placed(rows_done, nseg * kSmx, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait_cluster(bar(B_ROWS), 0, abort_flag)) { ok = false; break; }
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
                     }
                     const int sv = it % NSV;
                     if (!mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag)) { ok = false; break; }
@@ -572,7 +585,9 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 if (!mbar_wait_warp(bar(B_XFREE), (seg - 1) & 1, abort_flag)) return false;
             }
             if constexpr (ROPE) {
-                load_q_rotated<PAIR, ROWS>(sm, p.q, pa.rope_q, sg.b, sg.kvh, sg.mblock, rows_total, G, N, p.Hq, st);
+                // the Q tile and, beside it, this rank's share of the unit's tree rows into the cache
+                rope_prologue<PAIR, ROWS>(sm, p.q, pa, N, p.Hq, p.Hkv, p.S_max, G, rows_total, sg.b, sg.kvh, sg.mblock, sg.S,
+                                          (cr * N) / ck, ((cr + 1) * N) / ck, st);
                 fence_async_smem();
                 mbar_arrive(bar(B_QFULL));
                 return true;
@@ -618,26 +633,20 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 // every S product of the previous segment has been consumed by now, so Q may be replaced
                 if (!load_q(sg, seg)) { ok = false; break; }
                 if constexpr (ROPE) {
-                    // The tree rows that this CTA's own steps will read, of all its segments at once (the producer runs
-                    // segments ahead): into the cache now, while the first tiles are on their way.  The producer holds
-                    // the tiles that contain them back until every softmax thread has counted itself in, once per such
-                    // segment.
-                    if (seg == 0) {
-                        SegIter sj = make_iter();
-                        Seg sh;
-                        int placed = 0;
-                        while (sj.next(sh)) {
-                            const int t_lo = max(0, sh.st0 * STEP - sh.S), t_hi = min(N, (sh.st0 + sh.n) * STEP - sh.S);
-                            if (t_hi <= t_lo) continue;
-                            place_tree_rows(pa, N, p.Hkv, p.S_max, sh.b, sh.kvh, sh.S, t_lo, t_hi, st);
-                            ++placed;
-                        }
-                        if (placed > 0) {
-                            __threadfence();                                          // the rows are in global memory ...
-                            asm volatile("fence.proxy.async.global;" ::: "memory");   // ... and ordered before the bulk copies that read them
-                            atomicAdd(const_cast<int*>(rows_done), placed);
-                        }
+                    // Each rank of the cluster has just put its share of the unit's N tree rows into the cache (beside its Q
+                    // tile).  The ranks whose steps contain the rows (the last, at most the last two) hold those tiles back
+                    // until every rank has said that its share is in global memory: fence, meeting of this CTA's softmax
+                    // threads, then one arrival per rank on that rank's barrier.
+                    __threadfence();                                          // the rows are in global memory ...
+                    asm volatile("fence.proxy.async.global;" ::: "memory");   // ... and ordered before bulk copies that read them
+                    mbar_arrive(bar(B_SEGSYNC));
+                    if (!cl_waited) { cluster_wait(); cl_waited = true; }     // the peers' barriers exist
+                    if (st < ck) {
+                        if (!mbar_wait(bar(B_SEGSYNC), sx & 1, abort_flag)) { ok = false; }
+                        else mbar_arrive_peer(dsmem_addr(bar(B_ROWS), (uint32_t)st));
                     }
+                    ++sx;
+                    if (__any_sync(0xffffffffu, !ok)) { ok = false; break; }
                 }
 
                 const int row = sg.mblock * 128 + lrow;          // query row within the kv head's G*N rows
@@ -910,6 +919,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         // there without polling); then rank r merges rows [r*rp, (r+1)*rp) of all k partials through distributed
         // shared memory and writes them out. ----
         __syncwarp();
+        if (!cl_waited) { cluster_wait(); cl_waited = true; }     // (fused rotary embedding: the start-up phase, warps 0-3)
         cluster_sync_all();
         if (warp == 1) {
             // every thread of the CTA is past its last tensor-memory access: give the columns back now, beside the
@@ -1135,8 +1145,7 @@ cudaError_t init_attn_tc5() {
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
         if (e != cudaSuccess) return e;
     }
-    const void* rope_kernels[4] = {(const void*)attn_tc5_kernel<true, false, false, true>, (const void*)attn_tc5_kernel<false, false, false, true>,
-                                   (const void*)attn_tc5_kernel<true, true, false, true>, (const void*)attn_tc5_kernel<false, true, false, true>};
+    const void* rope_kernels[2] = {(const void*)attn_tc5_kernel<true, true, false, true>, (const void*)attn_tc5_kernel<false, true, false, true>};
     for (const void* k : rope_kernels) {
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ALLOC);
         if (e != cudaSuccess) return e;
@@ -1196,13 +1205,8 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
         auto launch_rope = [&](auto kernel, int cluster) {
             return launch_pdl(kernel, dim3(grid), dim3(kThreads), SMEM_ALLOC, st, cluster, *a.k_map, *a.v_map, p, ra);
         };
-        if (ck > 0) err = pair ? launch_rope(attn_tc5_kernel<true, true, false, true>, ck) : launch_rope(attn_tc5_kernel<false, true, false, true>, ck);
-        else err = pair ? launch_rope(attn_tc5_kernel<true, false, false, true>, 0) : launch_rope(attn_tc5_kernel<false, false, false, true>, 0);
-        if (err != cudaSuccess) return err;
-        ++*n_launches;
-        if (ck > 0 || own_merge) return cudaSuccess;
-        err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p)
-                   : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 8), dim3(128), 0, st, 0, p);
+        if (ck <= 0) return cudaErrorInvalidValue;        // cluster form only: the caller asks attn_tc5_uses_clusters first
+        err = pair ? launch_rope(attn_tc5_kernel<true, true, false, true>, ck) : launch_rope(attn_tc5_kernel<false, true, false, true>, ck);
         if (err != cudaSuccess) return err;
         ++*n_launches;
         return cudaSuccess;

@@ -47,6 +47,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
+// The same wait for a barrier that threads of other CTAs of the cluster arrive on (acquire at cluster scope).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  long long limit = kWaitCycles) {
+    long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 63) == 63) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit) { *abort_flag = 1; return false; }
+        }
+    }
+}
 // Same, with a warp-uniform result (every lane of a converged warp calls it): the warp-collective
 // tcgen05.ld/st that follow must never be reached by only part of a warp.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
@@ -85,6 +105,16 @@ __device__ __forceinline__ float4 dsmem_ld4(uint32_t a) {
 }
 __device__ __forceinline__ float2 dsmem_ld2(uint32_t a) {
     float2 v; asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a) : "memory"); return v;
+}
+// The hardware cluster barrier in two halves: a warp arrives once and waits once per phase, all its lanes together
+// (a wait taken by one lane and later by the other 31 never returns); the wait may sit anywhere later in the warp's
+// path.  Relaxed arrival: what the peers must see, the initialised barriers, is published by fence.mbarrier_init.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+// One arrival on an mbarrier of another CTA of the cluster (address from dsmem_addr), ordered after this thread's
+// earlier accesses at cluster scope.
+__device__ __forceinline__ void mbar_arrive_peer(uint32_t peer_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(peer_bar) : "memory");
 }
 // Programmatic dependent launch: let the next kernel in the stream be scheduled / wait for the previous one.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
