@@ -585,9 +585,11 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 if (!mbar_wait_warp(bar(B_XFREE), (seg - 1) & 1, abort_flag)) return false;
             }
             if constexpr (ROPE) {
-                // the Q tile and, beside it, this rank's share of the unit's tree rows into the cache
+                // the Q tile and, beside it, this rank's share of the unit's tree rows into the cache (a rejected
+                // sequence, steps == 0, has no slots to write to: an empty share)
+                const int t_lo = (cr * N) / ck;
                 rope_prologue<PAIR, ROWS>(sm, p.q, pa, N, p.Hq, p.Hkv, p.S_max, G, rows_total, sg.b, sg.kvh, sg.mblock, sg.S,
-                                          (cr * N) / ck, ((cr + 1) * N) / ck, st);
+                                          t_lo, sg.steps > 0 ? ((cr + 1) * N) / ck : t_lo, st);
                 fence_async_smem();
                 mbar_arrive(bar(B_QFULL));
                 return true;

@@ -205,6 +205,53 @@ def test_fused_rope_attention_matches_rope_then_attention_of_the_oracle(B, N, Hq
     ctx.close()
 
 
+@pytest.mark.parametrize("split_form", [0, 1])
+def test_fused_rope_attention_leaves_a_sequence_that_does_not_fit_alone(split_form):
+    """kv_len + N > S_max for one sequence: its cache rows stay as they were (nothing is written past its slots), its
+    output is zero with lse = -inf, the status word says so, and the other sequence is served as usual."""
+    from paper_2509_15235_b200 import binding
+    import gpu_util as gu
+    B, N, Hq, Hkv, D, S_max = 2, 24, 4, 4, 128, 512
+    kv_len = np.array([S_max - N + 3, 300], dtype=np.int32)           # sequence 0 would need 3 slots beyond its cache
+    rng = np.random.Generator(np.random.Philox(977))
+    q = synth.normal_bf16((B, N, Hq, D), 811); k = synth.normal_bf16((B, N, Hkv, D), 812)
+    v = synth.normal_bf16((B, N, Hkv, D), 813)
+    kc = synth.normal_bf16((B, Hkv, S_max, D), 814); vc = synth.normal_bf16((B, Hkv, S_max, D), 815)
+    parents = np.stack([synth.draw_tree(N, 5, 3, rng) for _ in range(B)])
+    mask, depth, _ = oracle.tree_mask(parents)
+    positions = (kv_len[:, None] + depth).astype(np.int32)
+    theta, scale = 1e4, 1.0 / np.sqrt(D)
+    o_q, o_k, o_v, skipped = oracle.rope_rows(q, k, v, positions, kv_len, kc, vc, theta)
+    assert skipped == 1
+    want, want_lse = oracle.tree_attn(o_q[1:], o_k[1:], o_v[1:], kv_len[1:], mask[1:], scale)
+
+    ctx = binding.VerifyContext(B, N, Hq, Hkv, D, S_max, 1)
+    if split_form:
+        ctx.ctx_set_option(binding.OPT_SPLIT_FORM, split_form)
+    # the caches sit in the middle of one allocation whose margins must come back untouched as well
+    pad = 64 * D
+    kbuf = torch.full((B * Hkv * S_max * D + 2 * pad,), 1.5, dtype=torch.bfloat16, device="cuda")
+    vbuf = torch.full_like(kbuf, 2.5)
+    kd = kbuf[pad:-pad].view(B, Hkv, S_max, D); vd = vbuf[pad:-pad].view(B, Hkv, S_max, D)
+    kd.copy_(gu.bf16_dev(kc)); vd.copy_(gu.bf16_dev(vc))
+    ctx.cache_register(0, kd, vd)
+    table = ctx.rope_table_build(gu.i32_dev(positions), theta)
+    out = torch.full((B, N, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, Hq, N), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.tree_verify_attn_rope(0, gu.bf16_dev(q), gu.bf16_dev(k), gu.bf16_dev(v), table, gu.i32_dev(kv_len), gu.u64_dev(mask),
+                              scale, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.status_poll() == -4
+    assert (kbuf[:pad] == 1.5).all() and (kbuf[-pad:] == 1.5).all() and (vbuf[:pad] == 2.5).all() and (vbuf[-pad:] == 2.5).all()
+    assert np.array_equal(gu.bf16_bits(kd[0].contiguous()), kc[0]) and np.array_equal(gu.bf16_bits(vd[0].contiguous()), vc[0])
+    assert np.array_equal(gu.bf16_bits(vd[1].contiguous()), o_v[1])
+    o = out.float().cpu().numpy()
+    assert (o[0] == 0).all() and np.isneginf(lse[0].cpu().numpy()).all()
+    assert np.abs(o[1] - want[0]).max() <= 2e-2
+    assert np.abs(lse[1].cpu().numpy() - want_lse[0]).max() <= 2e-3
+    ctx.close()
+
+
 def test_fused_rope_attention_refuses_what_it_does_not_serve():
     from paper_2509_15235_b200 import binding
     ctx = binding.VerifyContext(1, 8, 2, 2, 64, 128, 1)            # head size 64: the generic kernel's territory
