@@ -197,8 +197,9 @@ int vispec_rope_table_bytes(const vispec_ctx* ctx, int B, int N, size_t* out /*h
  * rounding to bf16, v copied, both written to slots kv_len[b] + i of the registered caches exactly as
  * vispec_rope_tree_rows writes them.  Short calls (the form with one thread-block cluster per head) run as ONE
  * launch: every thread block rotates the q rows it needs on their way into shared memory (fp32 arithmetic from the
- * table's fp32 half; the rotated q is consumed by the score product only), and the blocks whose share of the cache
- * contains the tree's slots write those rows before they read them.  Long calls (work split evenly over the SMs)
+ * table's fp32 half; the rotated q is consumed by the score product only), and the blocks of a head's cluster each
+ * write a share of the tree's rows into the cache before the block whose part of the cache contains those slots reads
+ * them (a sequence with kv_len + N > S_max is left alone: nothing written, zero output, VISPEC_E_RANGE).  Long calls (work split evenly over the SMs)
  * run as two launches - the rotation kernel fed from the table, writing the rotated q into a scratch copy at the end
  * of the workspace, then the plain attention - because there the in-kernel rotation costs more than it saves.  Everything else (tree_mask, kv_len, out, lse,
  * status word, early prefix reads) as in vispec_tree_verify_attn; rope_table comes from vispec_rope_table_build

@@ -239,7 +239,7 @@ __device__ __noinline__ void rope_prologue(unsigned char* sm, const __nv_bfloat1
     for (int u = 0; u < 2; ++u)
         if (ps >= 0 && ps + HALF * u < nv) vx[u] = *v_src(ps + HALF * u);
     // (with 128 rows per unit the Q tile alone takes 96 registers per thread: there the rows are finished first; timed in
-    // one call on qwen7b: 16.3 against 17.6 us per layer of a step with both sets of loads in flight)
+    // one call on qwen7b: 18.7 against 20.1 us per layer of a step with both sets of loads in flight)
     auto finish_rows = [&]() {
         if (has_k) k_store(ps, klo, khi, cs);
 #pragma unroll
