@@ -643,6 +643,16 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             return r;
         };
 
+        if (PAIR && active) {
+            // block-diagonal P: a lane's row copy weighs only its own half's 64 tokens of a step; the columns of the
+            // other half are zero in both P buffers for the whole call, and nobody else writes them
+            uint32_t zero[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) zero[c] = 0u;
+            tmem_st16(lane_addr + COL_P + (half ^ 1) * 32 + ch * 16, zero);
+            tmem_st16(lane_addr + COL_P + 64 + (half ^ 1) * 32 + ch * 16, zero);
+            tmem_wait_st();
+        }
         if (active) {
             SegIter si = make_iter();
             Seg sg;
@@ -749,6 +759,9 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                             tmem_st32(lane_addr + COL_O + ch * 64 + c * 32, o);
                         }
                     }
+                    // P[bs] is free once the PV product of step it-2 has completed: as a rule it has, long ago, and one test
+                    // issued here, ahead of the exponentials, says so without a wait after them
+                    const bool p_free = it < 2 || mbar_test(bar(B_PVDONE + bs), ((it >> 1) - 1) & 1);
                     // P = exp2(scale * s - m_ref) as bf16 pairs (column c of P holds tokens 2c, 2c+1)
                     uint32_t pd[NC / 2];
                     if (valid) {
@@ -768,18 +781,14 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                         for (int c = 0; c < NC / 2; ++c) pd[c] = 0u;
                     }
                     if (row_valid) has_o = true;
-                    // P[bs] is free once the PV product of step it-2 has completed
                     if (it >= 2) {
-                        if (!mbar_wait_warp(bar(B_PVDONE + bs), ((it >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+                        if (!__all_sync(0xffffffffu, p_free) &&
+                            !mbar_wait_warp(bar(B_PVDONE + bs), ((it >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                     }
                     if (PAIR) {
-                        // block-diagonal P: the row weighs only its own half's tokens, the other 32 columns are zero
-                        uint32_t zero[16];
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) zero[c] = 0u;
+                        // block-diagonal P: the row weighs only its own half's tokens (the other 32 columns stay zero)
                         tmem_st16(lane_addr + COL_P + bs * 64 + half * 32 + ch * 16, pd);
-                        tmem_st16(lane_addr + COL_P + bs * 64 + (half ^ 1) * 32 + ch * 16, zero);
                     } else {
                         tmem_st32(lane_addr + COL_P + bs * 64 + ch * 32, pd);
                     }
