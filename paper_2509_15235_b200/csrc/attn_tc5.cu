@@ -49,8 +49,14 @@
 // write come after that wait.
 //
 // Every wait on an mbarrier is bounded; on a timeout the CTA records VISPEC_E_TIMEOUT, drains its own
-// copies, frees its TMEM and returns.  The cluster form's two hardware cluster barriers are reached by every
-// thread of every CTA of the cluster (all other waits being bounded), so they end.
+// copies, frees its TMEM and returns.  The cluster form's hardware cluster barriers (two; three phases with the
+// fused rotary embedding, whose first is arrived at after set-up and waited for by whole warps before their first
+// signal to a peer) are reached by every thread of every CTA of the cluster (all other waits being bounded), so
+// they end.
+//
+// Fused rotary embedding (ROPE instantiations, cluster form, contiguous caches): each rank of a unit's cluster
+// rotates and places its share of the unit's N tree rows beside its (rotating) Q load and tells every rank; the
+// producers hold back the tiles that contain those slots until all ranks have told.
 #include <cuda_bf16.h>
 #include <cstdio>
 #include <cstdlib>
