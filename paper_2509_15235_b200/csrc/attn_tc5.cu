@@ -116,11 +116,12 @@ static_assert(SMEM_ALLOC <= 232448, "over the 227 KB a CTA may have");
 // masked like any slot past the end.  Not inlined, so that it stays out of the kernel's register budget, and
 // everything by value, so that the caller's counters stay in registers.  Returns steps issued in full | K-only
 // step << 28 | a wait gave up << 29 | has waited for the preceding kernel << 30 (the same in every lane).
-constexpr int kTabRing = 8, kTabAhead = 6;     // steps held in the ring / steps a copy is issued ahead
+constexpr int kTabRing = 4, kTabAhead = 3;     // steps held in a ring / steps a copy is issued ahead (two rings of
+                                               // 128 bytes: the K producer's and, where V has its own warp, the V producer's)
 __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensorMap* k_map, const CUtensorMap* v_map,
                                                int b, int kvh, int st0, int n, int S, uint32_t base, uint32_t bars,
                                                uint32_t ring, volatile int* abort_flag, uint64_t pol, int it,
-                                               bool waited, int lane) {
+                                               bool waited, int lane, int which /* 0: K and V, 1: K only, 2: V only */) {
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     const int nsub = STEP / p.page_rows;
     const uint32_t sub_bytes = (uint32_t)p.page_rows * 128u;
@@ -156,25 +157,29 @@ __device__ __noinline__ uint32_t produce_paged(const PagedArgs p, const CUtensor
         const uint32_t tx = (uint32_t)__popc(__ballot_sync(0xffffffffu, load)) * sub_bytes * 2u;
         const int sk = it % NSK, sv = it % NSV;
         bool w = true;
-        if (lane == 0) {
-            w = mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag);
-            if (w) mbar_expect_tx(bar(B_KFULL + sk), tx);
+        if (which != 2) {
+            if (lane == 0) {
+                w = mbar_wait(bar(B_KEMPTY + sk), ((it / NSK) & 1) ^ 1, abort_flag);
+                if (w) mbar_expect_tx(bar(B_KFULL + sk), tx);
+            }
+            w = __shfl_sync(0xffffffffu, w, 0);                          // the byte count is posted before any lane copies
+            if (!w) { fail = 2u << 28; break; }
+            if (load) {
+                tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 0, c1, c2, pol);
+                tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 64, c1, c2, pol);
+            }
         }
-        w = __shfl_sync(0xffffffffu, w, 0);                              // the byte count is posted before any lane copies
-        if (!w) { fail = 2u << 28; break; }
-        if (load) {
-            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 0, c1, c2, pol);
-            tma_load_3d(base + SMEM_K + sk * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, k_map, bar(B_KFULL + sk), 64, c1, c2, pol);
-        }
-        if (lane == 0) {
-            w = mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag);
-            if (w) mbar_expect_tx(bar(B_VFULL + sv), tx);
-        }
-        w = __shfl_sync(0xffffffffu, w, 0);
-        if (!w) { fail = 3u << 28; break; }
-        if (load) {
-            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 0, c1, c2, pol);
-            tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 64, c1, c2, pol);
+        if (which != 1) {
+            if (lane == 0) {
+                w = mbar_wait(bar(B_VEMPTY + sv), ((it / NSV) & 1) ^ 1, abort_flag);
+                if (w) mbar_expect_tx(bar(B_VFULL + sv), tx);
+            }
+            w = __shfl_sync(0xffffffffu, w, 0);
+            if (!w) { fail = (which == 2 ? 2u : 3u) << 28; break; }      // (V only: nothing of this step was issued)
+            if (load) {
+                tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 0, c1, c2, pol);
+                tma_load_3d(base + SMEM_V + sv * STAGE_BYTES + HALF_BYTES + lane * sub_bytes, v_map, bar(B_VFULL + sv), 64, c1, c2, pol);
+            }
         }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");                     // nothing of this segment stays in flight
@@ -342,7 +347,12 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     static_assert(!ROPE || CL, "the fused rotary embedding exists in the cluster form only (the even split goes through the rotation kernel)");
     constexpr int ROWS = PAIR ? 64 : 128;      // distinct query rows per CTA
     constexpr int NC = PAIR ? 32 : 64;         // tokens of a step one softmax thread handles (two threads per row)
-    constexpr bool SPLIT_V = PAIR && !PAGED;   // the V ring has a producer thread of its own (the spare warp's lane 0)
+    // The V ring can have a producer of its own, the spare warp (its lane 0; paged: all of it).  With at most 64 rows per
+    // unit it always has; with 128 only for pools of 16-row blocks, where one warp issuing a step's 32 copies is what
+    // holds the call back (larger blocks lose 1 % with two producers, like the contiguous cache).
+    constexpr bool SPLIT_V = PAIR || PAGED;
+    bool split_v = PAIR;
+    if constexpr (PAGED && !PAIR) split_v = pa.page_rows <= 16;
     extern __shared__ __align__(1024) unsigned char sm[];
     // the schedule hangs on kv_len, and a CTA that starts after its predecessor kernel has ended hangs on the
     // schedule: the load goes out first
@@ -436,9 +446,9 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             Seg sg;
             if constexpr (PAGED) {
                 while (ok && si.next(sg)) {
-                    const uint32_t r = produce_paged(pa, &k_map, &v_map, sg.b, sg.kvh, sg.st0, sg.n, sg.S, base, bars, base + SMEM_TABRING, abort_flag, pol, it, waited, lane);
+                    const uint32_t r = produce_paged(pa, &k_map, &v_map, sg.b, sg.kvh, sg.st0, sg.n, sg.S, base, bars, base + SMEM_TABRING, abort_flag, pol, it, waited, lane, split_v ? 1 : 0);
                     const int done = (int)(r & 0x0fffffffu);
-                    it += done; nv += done; nk += done + (int)((r >> 28) & 1u);
+                    it += done; nv += split_v ? 0 : done; nk += done + (int)((r >> 28) & 1u);
                     ok = !((r >> 29) & 1u);
                     waited = (r >> 30) & 1u;
                 }
@@ -484,7 +494,25 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         // Measured in one call, one thread against two: 17.70 -> 17.50 us per layer on llava7b, 17.11 -> 16.91 on
         // paper_tree, 71.4 -> 71.0 on llava13b_b4; with 128 rows per unit the two threads lose 1 % (16.43 -> 16.59 on
         // qwen7b, 63.3 -> 63.8 on qwen3b_S32768_N16_B8), so those keep the single producer.
-        if (SPLIT_V && lane == 0 && active) {
+        if constexpr (SPLIT_V && PAGED) {
+            if (active && split_v) {
+                const uint64_t pol = l2_evict_first_policy();
+                bool waited = !p.early, ok = true;
+                int it = 0;
+                SegIter si = make_iter();
+                Seg sg;
+                while (ok && si.next(sg)) {
+                    const uint32_t r = produce_paged(pa, &k_map, &v_map, sg.b, sg.kvh, sg.st0, sg.n, sg.S, base, bars, base + SMEM_TABRING + 128, abort_flag, pol, it, waited, lane, 2);
+                    it += (int)(r & 0x0fffffffu);
+                    ok = !((r >> 29) & 1u);
+                    waited = (r >> 30) & 1u;
+                }
+                if (*abort_flag && lane == 0) {
+                    volatile int never = 0;
+                    for (int u = max(0, it - NSV); u < it; ++u) mbar_wait(bar(B_VFULL + u % NSV), (u / NSV) & 1, &never);
+                }
+            }
+        } else if (SPLIT_V && lane == 0 && active) {
             const uint64_t pol = l2_evict_first_policy();
             bool waited = !p.early;
             int it = 0;
