@@ -24,8 +24,9 @@
 //   warp 1     issuer (one thread) of S = Q K^T as 128x128x16 tcgen05.mma; owns the TMEM allocation
 //   warp 2     issuer (one thread) of O += P V; the two chains wait on different barriers, so each has its own
 //              thread and neither's waits delay the other's instructions
-//   warp 3     derives the schedule from kv_len; with at most 64 rows per unit and a contiguous cache its lane 0
-//              then produces the V ring, so that warp 0's K copies never queue behind a wait for a V stage
+//   warp 3     derives the schedule from kv_len; with at most 64 rows per unit (its lane 0; the whole warp on a paged
+//              cache) and on pools of 16-row blocks it then produces the V ring, so that warp 0's K copies never
+//              queue behind a wait for a V stage
 //   warps 4-11 softmax: thread <-> TMEM lane; warps w and w+4 share the same 32 accumulator rows and each takes
 //              half of a step's columns (the row maximum is exchanged through shared memory), so a row costs
 //              no shuffles; they also load Q at the start of every segment and run the segment epilogue
