@@ -267,7 +267,7 @@ __device__ __noinline__ void rope_prologue(unsigned char* sm, const __nv_bfloat1
     float4 tab[PITEMS][4];
 #pragma unroll
     for (int k = 0; k < PITEMS; ++k) {
-        const int row = mblock * 128 + (st >> 3) + 32 * k;
+        const int row = mblock * ROWS + (st >> 3) + 32 * k;
         lo[k] = make_uint4(0, 0, 0, 0); hi[k] = lo[k];
 #pragma unroll
         for (int j = 0; j < 4; ++j) tab[k][j] = make_float4(1.f, 0.f, 1.f, 0.f);
@@ -652,7 +652,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             uint4 v[ITEMS];
 #pragma unroll
             for (int k = 0; k < ITEMS; ++k) {
-                const int row = sg.mblock * 128 + (st >> 4) + 16 * k;
+                const int row = sg.mblock * ROWS + (st >> 4) + 16 * k;
                 v[k] = make_uint4(0, 0, 0, 0);
                 if (row < rows_total) {
                     const int node = row / G, head = sg.kvh * G + row % G;
@@ -714,7 +714,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     if (__any_sync(0xffffffffu, !ok)) { ok = false; break; }
                 }
 
-                const int row = sg.mblock * 128 + lrow;          // query row within the kv head's G*N rows
+                const int row = sg.mblock * ROWS + lrow;         // query row within the kv head's G*N rows
                 const bool row_ok = row < rows_total;
                 const int node = row_ok ? row / G : 0, head = sg.kvh * G + (row_ok ? row % G : 0);
                 const int S = sg.S, total = S + N;
@@ -1009,7 +1009,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                     const int item = item0 + e * kSmx;
                     const int c4 = item / nrows, lr = row0 + (item - c4 * nrows);
                     c4s[e] = c4;
-                    grows[e] = (item < nrows * 32) ? cl_seg.mblock * 128 + lr : rows_total;
+                    grows[e] = (item < nrows * 32) ? cl_seg.mblock * ROWS + lr : rows_total;
 #pragma unroll
                     for (int j = 0; j < KM; ++j) {
                         ml[e][j] = make_float2(-INFINITY, 0.f);
@@ -1162,11 +1162,12 @@ static int query_max_clusters(bool pair, int k) {
 }
 
 // Cluster size for the cluster form, or 0 when the even split with partials in global memory serves better:
-// one cluster per unit, all clusters co-resident, and three quarters of the SMs in use (three fifths for short calls).
-static int tc5_cluster_size(const AttnArgs& a, int units) {
+// one cluster per unit, all clusters co-resident.  `pair`: units of at most 64 rows in the duplicated-row layout,
+// n_mblocks of them per kv head.  *est_us: the estimate of the form it returns.
+static int tc5_cluster_size(const AttnArgs& a, bool pair, int n_mblocks, double* est_us = nullptr) {
+    const int units = a.B * a.Hkv * n_mblocks;
+    if (est_us) *est_us = 1e30;
     if (a.tc5_path == 1 || a.tc5_path == 3) return 0;
-    const int rows_total = (a.Hq / a.Hkv) * a.N;
-    const bool pair = rows_total <= 64;
     int best = 0;
     for (int k = 1; k <= 8; ++k)
         if (units * k <= a.sm_count && g_max_clusters[pair][k] >= units) best = k;
@@ -1179,21 +1180,46 @@ static int tc5_cluster_size(const AttnArgs& a, int units) {
     // head read the same tiles, so only one in n_mblocks comes from HBM), and 0.25 per partial a unit is merged
     // from.  The host knows only the capacity S_max, not kv_len: the estimate is for full caches unless the caller
     // has given the length it expects (VISPEC_OPT_KV_LEN_HINT).
-    const int n_mblocks = pair ? 1 : (rows_total + 127) / 128;
     const int slots = (a.kv_len_hint > 0 && a.kv_len_hint + a.N < a.S_max) ? a.kv_len_hint + a.N : a.S_max;
     const double steps = (double)((slots + STEP - 1) / STEP), T = steps * units;
     const double n_c = (double)units * best, per_c = (double)(((slots + STEP - 1) / STEP + best - 1) / best);
     const double est_c = 11.0 + per_c * fmax(1.2, n_c * 0.0125 / n_mblocks);
     const double n_e = fmin((double)a.sm_count, fmax(1.0, T / 2.0));
     const double est_e = 14.0 + (T / n_e) * fmax(1.2, n_e * 0.00973 / n_mblocks) + 0.25 * (n_e / units);
+    if (est_us) *est_us = fmin(est_c, est_e);
     return est_c <= est_e ? best : 0;
+}
+
+// Row layout of a call.  At most 64 query rows per kv head: one unit of 64 rows, rows duplicated over the two lane
+// halves.  More: blocks of 128 rows, lane = row - unless that leaves most of the GPU idle (few sequences and kv
+// heads, rows just over 64: one cluster of at most 8 CTAs per unit is all the cluster form can use): then blocks of 64
+// rows in the duplicated layout make twice the units, and a step of such a unit costs its softmax threads half the
+// columns (measured per step and CTA: 0.9 against 1.4-1.8 us), at the price of every K/V tile crossing from L2 twice as
+// often and half of each product computed for nothing.  Taken when both layouts would run as clusters and the
+// estimate (steps of the busiest CTA at those rates) says a twentieth less or better.
+struct Tc5Layout { bool pair; int rows, n_mblocks, ck; };
+static Tc5Layout tc5_layout(const AttnArgs& a) {
+    const int rows_total = (a.Hq / a.Hkv) * a.N;
+    Tc5Layout full = {rows_total <= 64, rows_total <= 64 ? 64 : 128, rows_total <= 64 ? 1 : (rows_total + 127) / 128, 0};
+    full.ck = tc5_cluster_size(a, full.pair, full.n_mblocks);
+    if (full.pair || full.ck == 0 || a.tc5_path != 0) return full;
+    Tc5Layout half = {true, 64, (rows_total + 63) / 64, 0};
+    half.ck = tc5_cluster_size(a, true, half.n_mblocks);
+    if (half.ck == 0) return full;
+    const int slots = (a.kv_len_hint > 0 && a.kv_len_hint + a.N < a.S_max) ? a.kv_len_hint + a.N : a.S_max;
+    const int steps = (slots + STEP - 1) / STEP;
+    auto est = [&](const Tc5Layout& l, double step_us) {
+        const double n_c = (double)a.B * a.Hkv * l.n_mblocks * l.ck;
+        return 11.0 + (double)((steps + l.ck - 1) / l.ck) * fmax(step_us, n_c * 0.0125 / l.n_mblocks);
+    };
+    return est(half, 0.95) < 0.95 * est(full, full.n_mblocks > 1 ? 1.7 : 1.45) ? half : full;
 }
 
 bool attn_tc5_supports(const AttnArgs& a) {
     if (!(a.D == 128 && a.k_map && a.v_map && a.B > 0 && a.B <= kMaxB)) return false;
     const int rows_total = (a.Hq / a.Hkv) * a.N;
     const int rows = rows_total <= 64 ? 64 : 128;
-    const long long n_mblocks = rows_total <= 64 ? 1 : (rows_total + 127) / 128;
+    const long long n_mblocks = (rows_total + 63) / 64;          // the most either layout makes
     const long long t_max = (long long)a.B * a.Hkv * n_mblocks * ((a.S_max + STEP - 1) / STEP);
     if (t_max * a.sm_count >= (1ll << 31)) return false;
     if (!(a.scale > 0.f)) return false;       // the kernel takes the maximum before scaling
@@ -1223,21 +1249,15 @@ cudaError_t init_attn_tc5() {
     return cudaFuncSetAttribute(attn_tc5_merge_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
 }
 
-bool attn_tc5_uses_clusters(const AttnArgs& a) {
-    const int rows_total = (a.Hq / a.Hkv) * a.N;
-    const int n_mblocks = rows_total <= 64 ? 1 : (rows_total + 127) / 128;
-    return tc5_cluster_size(a, a.B * a.Hkv * n_mblocks) > 0;
-}
+bool attn_tc5_uses_clusters(const AttnArgs& a) { return tc5_layout(a).ck > 0; }
 
 cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches) {
     *n_launches = 0;
-    const int rows_total = (a.Hq / a.Hkv) * a.N;
-    const bool pair = rows_total <= 64;
-    const int rows = pair ? 64 : 128;
-    const int n_mblocks = pair ? 1 : (rows_total + 127) / 128;
+    const Tc5Layout lay = tc5_layout(a);
+    const bool pair = lay.pair;
+    const int rows = lay.rows, n_mblocks = lay.n_mblocks, ck = lay.ck;
     const int units = a.B * a.Hkv * n_mblocks;
     const long long t_max = (long long)units * ((a.S_max + STEP - 1) / STEP);
-    const int ck = tc5_cluster_size(a, units);
     const int grid = ck > 0 ? units * ck : (int)(t_max < a.sm_count ? t_max : a.sm_count);
 
     Tc5Params p = {};

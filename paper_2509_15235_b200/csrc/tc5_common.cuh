@@ -396,7 +396,7 @@ __device__ __noinline__ void merge_unit(const MergeArgs m, int T, int geff, int 
                                         int mblock, int st, int nthreads) {
     for (int item = st; item < ROWS * 8; item += nthreads) {
         const int cw = item / ROWS, lrow = item - cw * ROWS;
-        const int row = mblock * 128 + lrow;
+        const int row = mblock * ROWS + lrow;
         if (row >= m.rows_total) continue;
         merge_row_cols<ROWS>(m.part_o, m.part_ml, m.out, m.lse, T, geff, ub, c0, c1, b, row / m.G, kvh * m.G + row % m.G,
                              m.Hq, m.N, lrow, cw);
@@ -449,7 +449,7 @@ attn_tc5_merge_kernel(const Tc5Params p) {
     const int kvh = uib / p.n_mblocks, mblock = uib - kvh * p.n_mblocks;
     const int lrow = (blockIdx.y >> 1) * 32 + lane;
     const int cw = (blockIdx.y & 1) * 4 + warp;         // which 16 output columns
-    const int row = mblock * 128 + lrow;
+    const int row = mblock * ROWS + lrow;
     if (row >= G * N) return;
     const int node = row / G, head = kvh * G + row % G;
 
