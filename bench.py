@@ -40,11 +40,11 @@ FALLBACK_HBM_GBS = 6650.0
 # (dram__bytes_read.sum + dram__bytes_write.sum, two launches averaged).  A figure is only valid for the kernel it was
 # taken on: set an entry to None when the attention kernel changes and take the counters again.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    "llava7b": 66_200_000,                # 65.58 MB read + 0.63 MB written
-    "llava13b_b4": 335_570_000,           # 330.25 MB read + 5.32 MB written
-    "qwen3b_S32768_N16_B8": 274_270_000,  # attention launch only (270.08 + 4.19 MB); the merge kernel is its own launch
+    "llava7b": 66_180_000,                # 65.58 MB read + 0.61 MB written
+    "llava13b_b4": 335_860_000,           # 330.23 MB read + 5.63 MB written
+    "qwen3b_S32768_N16_B8": 274_060_000,  # attention launch only (270.09 + 3.97 MB); the merge kernel is its own launch
     "qwen3b_S8192_N60_B4": 35_150_000,    # four row blocks per kv head share their tiles through L2
-    "qwen7b": 7_585_000,
+    "qwen7b": 7_580_000,                  # seven row blocks per kv head share their tiles through L2
 }
 FALLBACK_BF16_TFLOPS = 1400.0             # sustained figure of the fallback measurement
 EXP_PER_CLK_PER_SM = 16                   # special-function lanes of one SM (4 per scheduler)
