@@ -1164,7 +1164,7 @@ static int query_max_clusters(bool pair, int k) {
 // Cluster size for the cluster form, or 0 when the even split with partials in global memory serves better:
 // one cluster per unit, all clusters co-resident.  `pair`: units of at most 64 rows in the duplicated-row layout,
 // n_mblocks of them per kv head.  *est_us: the estimate of the form it returns.
-static int tc5_cluster_size(const AttnArgs& a, bool pair, int n_mblocks, double* est_us = nullptr) {
+static int tc5_cluster_size(const AttnArgs& a, bool pair, int n_mblocks, double* est_us = nullptr, bool clusters_if_possible = false) {
     const int units = a.B * a.Hkv * n_mblocks;
     if (est_us) *est_us = 1e30;
     if (a.tc5_path == 1 || a.tc5_path == 3) return 0;
@@ -1172,7 +1172,7 @@ static int tc5_cluster_size(const AttnArgs& a, bool pair, int n_mblocks, double*
     for (int k = 1; k <= 8; ++k)
         if (units * k <= a.sm_count && g_max_clusters[pair][k] >= units) best = k;
     if (best == 0) return 0;
-    if (a.tc5_path == 2) return best;
+    if (a.tc5_path == 2 || clusters_if_possible) return best;
     // Both forms, estimated in microseconds from what was measured over the workloads (the long-response sweep
     // cells, the 7B and 13B shapes): a fixed part (11 for the cluster form, 14 for the even split with its partials
     // and second phase), the steps of the busiest CTA at 1.2 per step or at the HBM share of that many CTAs (64 KB
@@ -1185,12 +1185,14 @@ static int tc5_cluster_size(const AttnArgs& a, bool pair, int n_mblocks, double*
     const double n_c = (double)units * best, per_c = (double)(((slots + STEP - 1) / STEP + best - 1) / best);
     const double est_c = 11.0 + per_c * fmax(1.2, n_c * 0.0125 / n_mblocks);
     const double n_e = fmin((double)a.sm_count, fmax(1.0, T / 2.0));
-    const double est_e = 14.0 + (T / n_e) * fmax(1.2, n_e * 0.00973 / n_mblocks) + 0.25 * (n_e / units);
+    // (merge: 0.25 per piece of a unit; from four pieces on the fine-grained merge kernel, 1 + 0.055 per piece)
+    const double pieces = n_e / units;
+    const double est_e = 14.0 + (T / n_e) * fmax(1.2, n_e * 0.00973 / n_mblocks) + (pieces >= 4.0 ? 1.0 + 0.055 * pieces : 0.25 * pieces);
     // (units of several row blocks per kv head in small clusters: measured over the sweep, the even split's steps come
     // out dearer than the estimate there - 54.8 against 52.6 us on qwen3b_S8192_N60_B8, 96.1 against 92.4 on
     // qwen3b_S16384_N128_B4 - so the clusters get a tenth of tolerance)
     const double tol = (n_mblocks > 1 && best <= 4) ? 1.1 : 1.0;
-    if (est_us) *est_us = fmin(est_c, est_e);
+    if (est_us) *est_us = est_c <= tol * est_e ? est_c : est_e;
     return est_c <= tol * est_e ? best : 0;
 }
 
@@ -1205,10 +1207,11 @@ struct Tc5Layout { bool pair; int rows, n_mblocks, ck; };
 static Tc5Layout tc5_layout(const AttnArgs& a) {
     const int rows_total = (a.Hq / a.Hkv) * a.N;
     Tc5Layout full = {rows_total <= 64, rows_total <= 64 ? 64 : 128, rows_total <= 64 ? 1 : (rows_total + 127) / 128, 0};
-    full.ck = tc5_cluster_size(a, full.pair, full.n_mblocks);
-    if (full.pair || full.ck == 0 || a.tc5_path != 0) return full;
+    double est_full = 0.0;
+    full.ck = tc5_cluster_size(a, full.pair, full.n_mblocks, &est_full);
+    if (full.pair || a.tc5_path != 0) return full;
     Tc5Layout half = {true, 64, (rows_total + 63) / 64, 0};
-    half.ck = tc5_cluster_size(a, true, half.n_mblocks);
+    half.ck = tc5_cluster_size(a, true, half.n_mblocks, nullptr, true);     // (clusters or nothing: the even split gains nothing from smaller blocks)
     if (half.ck == 0) return full;
     const int slots = (a.kv_len_hint > 0 && a.kv_len_hint + a.N < a.S_max) ? a.kv_len_hint + a.N : a.S_max;
     const int steps = (slots + STEP - 1) / STEP;
@@ -1216,7 +1219,10 @@ static Tc5Layout tc5_layout(const AttnArgs& a) {
         const double n_c = (double)a.B * a.Hkv * l.n_mblocks * l.ck;
         return 11.0 + (double)((steps + l.ck - 1) / l.ck) * fmax(step_us, n_c * 0.0125 / l.n_mblocks);
     };
-    return est(half, 0.95) < 0.95 * est(full, full.n_mblocks > 1 ? 1.7 : 1.45) ? half : full;
+    if (full.ck > 0) return est(half, 0.95) < 0.95 * est(full, full.n_mblocks > 1 ? 1.7 : 1.45) ? half : full;
+    // 128-row blocks would go as an even split (its estimate: est_full); small clusters of 64-row blocks, whose fixed
+    // part measures 8 rather than 11 us, against that
+    return est(half, 0.95) - 3.0 < 0.95 * est_full ? half : full;
 }
 
 bool attn_tc5_supports(const AttnArgs& a) {
@@ -1248,9 +1254,13 @@ cudaError_t init_attn_tc5() {
     for (int k = 1; k <= 8; ++k) { g_max_clusters[0][k] = query_max_clusters(false, k); g_max_clusters[1][k] = query_max_clusters(true, k); }
     if (getenv("VISPEC_DEBUG")) for (int k = 1; k <= 8; ++k) fprintf(stderr, "vispec: cluster size %d: %d (rows > 64) / %d (rows <= 64) co-resident clusters\n", k, g_max_clusters[0][k], g_max_clusters[1][k]);
     // The merge blocks must be able to join an SM that an attention CTA has configured for maximum shared memory.
-    e = cudaFuncSetAttribute(attn_tc5_merge_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attn_tc5_merge_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    const void* merge_kernels[4] = {(const void*)attn_tc5_merge_kernel<64>, (const void*)attn_tc5_merge_kernel<128>,
+                                    (const void*)attn_tc5_merge_kernel<64, true>, (const void*)attn_tc5_merge_kernel<128, true>};
+    for (const void* k : merge_kernels) {
+        e = cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 bool attn_tc5_uses_clusters(const AttnArgs& a) { return tc5_layout(a).ck > 0; }
@@ -1313,8 +1323,12 @@ cudaError_t launch_attn_tc5(const AttnArgs& a, cudaStream_t st, int* n_launches)
     if (err != cudaSuccess) return err;
     ++*n_launches;
     if (own_merge) return cudaSuccess;
-    err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p)
-               : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 8), dim3(128), 0, st, 0, p);
+    if (grid >= 4 * units)        // units cut into many pieces: the fine-grained merge
+        err = pair ? launch_pdl(attn_tc5_merge_kernel<64, true>, dim3(units, 16), dim3(128), 0, st, 0, p)
+                   : launch_pdl(attn_tc5_merge_kernel<128, true>, dim3(units, 32), dim3(128), 0, st, 0, p);
+    else
+        err = pair ? launch_pdl(attn_tc5_merge_kernel<64>, dim3(units, 4), dim3(128), 0, st, 0, p)
+                   : launch_pdl(attn_tc5_merge_kernel<128>, dim3(units, 8), dim3(128), 0, st, 0, p);
     if (err != cudaSuccess) return err;
     ++*n_launches;
     return cudaSuccess;

@@ -388,6 +388,53 @@ __device__ __forceinline__ void merge_row_cols(const float4* __restrict__ part_o
         lse[((size_t)b * Hq + head) * N + node] = l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
 }
 
+// One (row, 4 output columns) of a unit, the merge kernel's piece: sixteen segments at a time with every load issued
+// before the first use (a unit cut over many CTAs - few sequences, long caches - is merged from dozens of partials,
+// and a round of loads is a memory round trip).
+template <int ROWS>
+__device__ __forceinline__ void merge_row_c4(const float4* __restrict__ part_o, const float2* __restrict__ part_ml,
+                                             __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int T, int geff,
+                                             int ub, int c0, int c1, int b, int node, int head, int Hq, int N,
+                                             int lrow, int c4) {
+    auto slot_of = [&](int c) { return cta_lo(c, T, geff) >= ub ? 2 * c : 2 * c + 1; };
+    float m_all = -INFINITY, l_all = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int cb = c0; cb <= c1; cb += 16) {
+        float2 ml[16];
+        float4 v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int c = cb + j;
+            ml[j] = make_float2(-INFINITY, 0.f);
+            v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c <= c1) {
+                const int slot = slot_of(c);
+                ml[j] = __ldcg(&part_ml[(size_t)slot * ROWS + lrow]);
+                v[j] = __ldcg(part_o + ((size_t)slot * 32 + c4) * ROWS + lrow);
+            }
+        }
+        float m_new = m_all;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) m_new = fmaxf(m_new, ml[j].x);
+        const float m_fin = (m_new == -INFINITY) ? 0.f : m_new;
+        const float a = exp2f(m_all - m_fin);                 // 0 while nothing has been accumulated
+        l_all *= a;
+        acc.x *= a; acc.y *= a; acc.z *= a; acc.w *= a;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float w = exp2f(ml[j].x - m_fin);           // 0 for a segment that saw nothing (or is absent)
+            l_all += ml[j].y * w;
+            acc.x += w * v[j].x; acc.y += w * v[j].y; acc.z += w * v[j].z; acc.w += w * v[j].w;
+        }
+        m_all = m_new;
+    }
+    const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+    *reinterpret_cast<uint2*>(out + (((size_t)b * N + node) * Hq + head) * D + c4 * 4) =
+        make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+    if (lse && c4 == 0)
+        lse[((size_t)b * Hq + head) * N + node] = l_all > 0.f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+}
+
 // The whole unit, by the softmax threads of the CTA that delivered the unit's last partial (thread st of nthreads).
 // Not inlined: its accumulators stay out of the attention kernel's register budget.
 struct MergeArgs { const float4* part_o; const float2* part_ml; __nv_bfloat16* out; float* lse; int Hq, G, N, rows_total; };
@@ -418,11 +465,15 @@ struct RopeArgs {
 struct PagedArgs { const int32_t* block_table; int table_stride, page_rows, num_blocks, Hkv, N, token_major; int* status;
                    int* unit_counters; };   // even split: arrivals per unit (all zero between calls); nullptr: a merge kernel follows
 
-// Merge of the partials of every unit that more than one CTA worked on.  Grid (unit, 2 * group of 32 rows +
-// half of the columns), 4 warps; lane <-> row, a warp sums 16 output columns over the unit's segments.
+// Merge of the partials of every unit that more than one CTA worked on, 4 warps per block, lane <-> row.  Two
+// shapes: grid (unit, 2 * group of 32 rows + half of the columns), a warp sums 16 output columns over the unit's
+// segments four at a time - for units cut into a few pieces; FINE: grid (unit, 8 * group of 32 rows + eighth of the
+// columns), a warp sums 4 output columns sixteen segments at a time - for units cut over many CTAs (few sequences, long
+// caches), where the rounds of loads are what the merge takes: qwen3b_S32768_N16_B1 (2 units over 148 CTAs) 42.7 ->
+// 29.1 us per layer, qwen3b_S32768_N60_B1 34.8 -> 31.8; with many units of two partials the coarse shape is 3 % faster.
 // The blocks are small so that they fit beside a resident attention CTA: they are launched early
 // (programmatic dependent launch) and must not keep the next layer's attention CTAs off the SMs.
-template <int ROWS>
+template <int ROWS, bool FINE = false>
 __global__ void __launch_bounds__(128)
 attn_tc5_merge_kernel(const Tc5Params p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -447,13 +498,14 @@ attn_tc5_merge_kernel(const Tc5Params p) {
     if (c0 == c1) return;                              // one CTA had the whole unit and wrote the output itself
     const int G = p.Hq / p.Hkv, N = p.N;
     const int kvh = uib / p.n_mblocks, mblock = uib - kvh * p.n_mblocks;
-    const int lrow = (blockIdx.y >> 1) * 32 + lane;
-    const int cw = (blockIdx.y & 1) * 4 + warp;         // which 16 output columns
+    const int lrow = (FINE ? blockIdx.y >> 3 : blockIdx.y >> 1) * 32 + lane;
+    const int cw = FINE ? (blockIdx.y & 7) * 4 + warp : (blockIdx.y & 1) * 4 + warp;    // which 4 (FINE) or 16 output columns
     const int row = mblock * ROWS + lrow;
     if (row >= G * N) return;
     const int node = row / G, head = kvh * G + row % G;
 
-    merge_row_cols<ROWS>(p.part_o, p.part_ml, p.out, p.lse, T, geff, ub, c0, c1, b, node, head, p.Hq, N, lrow, cw);
+    if (FINE) merge_row_c4<ROWS>(p.part_o, p.part_ml, p.out, p.lse, T, geff, ub, c0, c1, b, node, head, p.Hq, N, lrow, cw);
+    else merge_row_cols<ROWS>(p.part_o, p.part_ml, p.out, p.lse, T, geff, ub, c0, c1, b, node, head, p.Hq, N, lrow, cw);
 }
 
 // Launch with programmatic stream serialisation and, when cluster > 0, thread-block clusters of that size.
