@@ -49,8 +49,8 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {
 FALLBACK_BF16_TFLOPS = 1400.0             # sustained figure of the fallback measurement
 EXP_PER_CLK_PER_SM = 16                   # special-function lanes of one SM (4 per scheduler)
 # Workloads timed briefly after the headline (attention sweep only), each against its own binding roofline.
-OTHER_WORKLOADS = [("qwen7b", 28, False), ("llava13b_b4", 8, False), ("qwen3b_S8192_N16_B4", 16, False),
-                   ("qwen3b_S8192_N60_B4", 16, False), ("llava7b", 8, True)]
+OTHER_WORKLOADS = [("qwen7b", 28, False, 0), ("llava13b_b4", 8, False, 0), ("llava13b_b4", 8, False, 16),
+                   ("qwen3b_S8192_N16_B4", 16, False, 0), ("qwen3b_S8192_N60_B4", 16, False, 0), ("llava7b", 8, True, 0)]
 
 
 def parse_args():
@@ -407,11 +407,12 @@ class HostStep:
         self.s_out.synchronize()
 
 
-def time_other_workload(name, layers, redundant, device, min_seconds=0.4):
+def time_other_workload(name, layers, redundant, device, min_seconds=0.4, page_rows=0):
     """Attention sweep of one further workload (L layers, each its own cache pair, graph replay), timed for at least
     `min_seconds` with the clocks sampled meanwhile, against that workload's own binding roofline.  Trees and
     lengths come from the seeded generators; q/K/V are N(0,1) bf16 drawn on the device (timing only: these
-    workloads have their parity tests).  `redundant`: the image span of every head repeats one key (Sec. 4.1, Eq. 2)."""
+    workloads have their parity tests).  `redundant`: the image span of every head repeats one key (Sec. 4.1, Eq. 2).
+    `page_rows`: the caches are pools of blocks of that many slots, addressed through a block table in random order."""
     import torch
     from paper_2509_15235_b200 import binding, synth
     cfg = synth.get_config(name)
@@ -427,7 +428,12 @@ def time_other_workload(name, layers, redundant, device, min_seconds=0.4):
         v = torch.randn((B, Hkv, cfg.S_max, D), generator=g, device=dev, dtype=torch.bfloat16)
         if redundant:
             k[:, :, :cfg.n_image] = k[:, :, :1]
-        ctx.cache_register(l, k, v)
+        if page_rows:
+            k = k.view(B * (cfg.S_max // page_rows), page_rows, Hkv, D).permute(0, 2, 1, 3).contiguous()    # [blocks, Hkv, rows, D]
+            v = v.view(B * (cfg.S_max // page_rows), page_rows, Hkv, D).permute(0, 2, 1, 3).contiguous()
+            ctx.cache_register_paged(l, k, v, False)
+        else:
+            ctx.cache_register(l, k, v)
         ks.append(k); vs.append(v)
     q = torch.randn((L, B, N, Hq, D), generator=g, device=dev, dtype=torch.bfloat16)
     out = torch.empty_like(q)
@@ -437,9 +443,18 @@ def time_other_workload(name, layers, redundant, device, min_seconds=0.4):
     ctx.tree_mask_build(parents, mask)
     scale = 1.0 / math.sqrt(D)
 
+    block_table = None
+    if page_rows:
+        per = cfg.S_max // page_rows
+        perm = torch.randperm(B * per, generator=torch.Generator(device="cpu").manual_seed(4321))
+        block_table = perm.view(B, per).to(torch.int32).to(dev).contiguous()
+
     def sweep():
         for l in range(L):
-            ctx.tree_verify_attn(l, q[l], kv_len, mask, scale, out[l])
+            if page_rows:
+                ctx.tree_verify_attn_paged(l, q[l], kv_len, block_table, mask, scale, out[l])
+            else:
+                ctx.tree_verify_attn(l, q[l], kv_len, mask, scale, out[l])
 
     n0 = ctx.launch_count()
     sweep()
@@ -469,8 +484,9 @@ def time_other_workload(name, layers, redundant, device, min_seconds=0.4):
     status = ctx.status_poll()
     us = ms * 1e3 / (reps * L)
     sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
-    res = attention_roofline(cfg, tree["kv_len"], us, sm_count, NCU_TRAFFIC_BYTES_PER_LAUNCH.get(name) if not redundant else None)
-    res.update({"workload": name + ("+redundant_image_keys" if redundant else ""), "layers": L, "us_per_layer": us,
+    res = attention_roofline(cfg, tree["kv_len"], us, sm_count, NCU_TRAFFIC_BYTES_PER_LAUNCH.get(name) if not (redundant or page_rows) else None)
+    res.update({"workload": name + ("+redundant_image_keys" if redundant else "") + (f"+paged{page_rows}" if page_rows else ""),
+                "layers": L, "us_per_layer": us,
                 "sweeps": reps, "launches_per_call": launches_per_call, "status_word": status,
                 "kv_mb_per_layer": cfg.kv_bytes_per_layer(tree["kv_len"]) / 1e6,
                 "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "power_w_max")}})
@@ -733,7 +749,7 @@ def main():
                  "us_per_launch": sweep_us, "sweeps": sweep_reps})
     others = None
     if not args.no_others and not (args.paged or args.with_rope or args.layers):
-        others = [time_other_workload(n, l, r, local) for n, l, r in OTHER_WORKLOADS if not (n == cfg.name and not r)]
+        others = [time_other_workload(n, l, r, local, page_rows=pg) for n, l, r, pg in OTHER_WORKLOADS if not (n == cfg.name and not r and not pg)]
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
